@@ -1,0 +1,140 @@
+/*
+ * libstreamops -- the memory-bound streaming kernels Copy, Mul (scale), Add, Triad and Dot for
+ * NVIDIA B200 (sm_100a), behind a plain C ABI.
+ *
+ * The kernels are the five STREAM-style vector operations the paper evaluates (Table 1:
+ * "Copy", "Mul", "Add", "Triad", "Dot"; Section 5.2). The paper names them without printing a
+ * formula; each entry point below states the textbook definition it implements.
+ *
+ * Conventions for every stream_* entry point
+ *   - x, y, out are DEVICE pointers on the current device to dense, contiguous 1-D arrays of n
+ *     elements (out of Dot: one element). The caller owns them; the library never frees,
+ *     reallocates or keeps them.
+ *   - The call is asynchronous on `stream` (a cudaStream_t passed as a pointer; NULL is the
+ *     default stream). No call synchronises the host, copies to the host, or allocates, except
+ *     the one-time per-device workspace described under streamops_init.
+ *   - `scalar` is rounded once, to nearest-even, to the element type before use. Copy, Add and
+ *     Dot ignore it (one uniform signature).
+ *   - Arithmetic is IEEE-754 round-to-nearest-even in the element type, subnormals honoured,
+ *     one rounding per operation: Triad is a rounded multiply followed by a rounded add, never
+ *     a fused multiply-add. The four elementwise kernels therefore have exactly one correct
+ *     bit pattern per element (NaN payloads aside; Copy preserves every bit pattern).
+ *   - Pointers must be aligned to the element size; 16- or 32-byte alignment selects the
+ *     vector kernels, anything else runs the scalar kernel with identical results.
+ *   - out may be exactly x or exactly y (in place). Any other overlap of out with an input is
+ *     rejected with STREAMOPS_ERR_OVERLAP.
+ *   - n == 0 is valid and touches no element (Dot writes +0).
+ *   - Return value: a STREAMOPS_* status. Nothing throws, aborts or prints.
+ */
+#ifndef STREAMOPS_H
+#define STREAMOPS_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *streamops_stream_t; /* a cudaStream_t */
+
+enum streamops_status {
+    STREAMOPS_OK = 0,
+    STREAMOPS_ERR_NULL = 1,      /* a null pointer with n > 0 */
+    STREAMOPS_ERR_ALIGN = 2,     /* a pointer not aligned to the element size */
+    STREAMOPS_ERR_OVERLAP = 3,   /* out partially overlaps an input */
+    STREAMOPS_ERR_CUDA = 4,      /* a CUDA call failed; see streamops_last_cuda_error */
+    STREAMOPS_ERR_WORKSPACE = 5, /* the per-device workspace could not be created */
+    STREAMOPS_ERR_TIMEOUT = 6,   /* a bounded wait inside a bulk-copy kernel gave up */
+    STREAMOPS_ERR_ARG = 7        /* an argument outside its documented range */
+};
+
+enum streamops_op { STREAMOPS_COPY = 0, STREAMOPS_SCALE = 1, STREAMOPS_ADD = 2,
+                    STREAMOPS_TRIAD = 3, STREAMOPS_DOT = 4 };
+enum streamops_dtype { STREAMOPS_F32 = 0, STREAMOPS_F64 = 1 };
+
+/* Copy (Table 1, "Copy"): out[i] = x[i] for 0 <= i < n, bit for bit (NaN payloads, signed
+ * zeros and subnormals preserved). Moves 2*n*sizeof(T) bytes. */
+int stream_copy_f64(const double *x, double *out, double scalar, size_t n, streamops_stream_t stream);
+int stream_copy_f32(const float *x, float *out, double scalar, size_t n, streamops_stream_t stream);
+
+/* Mul (Table 1, "Mul"; exported as "scale"): out[i] = RN(s * x[i]), s = (T)scalar.
+ * Moves 2*n*sizeof(T) bytes. */
+int stream_scale_f64(const double *x, double *out, double scalar, size_t n, streamops_stream_t stream);
+int stream_scale_f32(const float *x, float *out, double scalar, size_t n, streamops_stream_t stream);
+
+/* Add (Table 1, "Add"): out[i] = RN(x[i] + y[i]). Moves 3*n*sizeof(T) bytes. */
+int stream_add_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
+int stream_add_f32(const float *x, const float *y, float *out, double scalar, size_t n, streamops_stream_t stream);
+
+/* Triad (Table 1, "Triad"): out[i] = RN(x[i] + RN(s * y[i])), s = (T)scalar; two roundings.
+ * Moves 3*n*sizeof(T) bytes. */
+int stream_triad_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
+int stream_triad_f32(const float *x, const float *y, float *out, double scalar, size_t n, streamops_stream_t stream);
+
+/* Dot (Table 1, "Dot"): out[0] = (T) sum_i x[i]*y[i]. out is a DEVICE pointer to one element;
+ * the result stays on the device. Products and sums are carried in double for both element
+ * types (a float*float product is exact in double) and rounded once to T at the end. The
+ * summation order is a fixed function of n and the tuning in force -- never of block arrival
+ * order or of the stream -- so repeated calls return identical bits. Accuracy: within relative
+ * 1e-12 (double) / 1e-5 (float) of the exactly rounded dot product for the documented
+ * workloads. Reads 2*n*sizeof(T) bytes. Uses one slot of the per-device workspace; at most
+ * STREAMOPS_DOT_SLOTS Dot calls may be in flight on one device at a time (slots are handed out
+ * round-robin; more concurrent calls than slots would share a slot and race). */
+int stream_dot_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
+int stream_dot_f32(const float *x, const float *y, float *out, double scalar, size_t n, streamops_stream_t stream);
+#define STREAMOPS_DOT_SLOTS 32
+
+/* One pass of the five kernels over three HOST arrays of n elements each, in the textbook
+ * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The three arrays are
+ * copied to the device, the five kernels above run on them, and the three arrays and the dot
+ * product are copied back; the call returns after the results are in host memory. a, b, c and
+ * dot_out are HOST pointers owned by the caller (pinned memory makes the copies asynchronous to
+ * each other; pageable memory works). Device buffers are allocated on the first call and reused
+ * while n does not grow; streamops_shutdown frees them. This is the end-to-end entry point for
+ * callers whose data lives on the host. */
+int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out);
+int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out);
+
+/* Creates the per-device state for `device` (SM count, the Dot workspace: partial sums, arrival
+ * tickets, an error flag; a few MiB). Optional: every entry point does it on first use for the
+ * current device. Allocates device memory, so call it outside stream capture. */
+int streamops_init(int device);
+
+/* Frees every per-device workspace and host-path buffer. The library can be used again after. */
+int streamops_shutdown(void);
+
+/* Tuning of one (op, dtype) pair: which kernel family and launch shape the entry point uses.
+ * Meant for benchmarking A/B runs; the defaults are the measured best on B200. Results of the
+ * elementwise kernels do not depend on it; Dot's summation order (hence its last bits) does. */
+typedef struct streamops_tuning {
+    int kind;           /* 0 = register-vector kernel (ld/st.global), 1 = bulk-copy (TMA) pipeline */
+    int vec_bytes;      /* kind 0: 16 or 32 (256-bit ld/st.global) */
+    int unroll;         /* kind 0: vectors per thread per array in flight: 1, 2 or 4 */
+    int threads;        /* threads per block: 128, 256 or 512 (kind 1: consumer threads) */
+    int blocks_per_sm;  /* persistent grid = blocks_per_sm * SMs; 0 = one block per tile */
+    int policy;         /* kind 0 cache-hint set, 0..4 (see streamops_policy_name) */
+    int contiguous;     /* 0 = tiles interleaved across blocks, 1 = one contiguous range per block */
+    int chunk_bytes;    /* kind 1: bytes per bulk copy per array (multiple of 16, <= 65536) */
+    int stages;         /* kind 1: ring depth, 2..8 */
+    int two_pass;       /* Dot only: 1 = second pass as its own launch, 0 = last block finishes */
+} streamops_tuning_t;
+
+int streamops_set_tuning(int op, int dtype, const streamops_tuning_t *t);
+int streamops_get_tuning(int op, int dtype, streamops_tuning_t *t);
+int streamops_reset_tuning(void);
+const char *streamops_policy_name(int policy);
+
+/* Reads the device error flag of the current device (a bounded wait that gave up sets it),
+ * after synchronising `stream`. Returns STREAMOPS_OK or STREAMOPS_ERR_TIMEOUT and clears it. */
+int streamops_check(streamops_stream_t stream);
+
+const char *streamops_status_string(int status);
+int streamops_last_cuda_error(void); /* the cudaError_t behind the last STREAMOPS_ERR_CUDA */
+
+/* Number of kernels this library has launched since it was loaded (all devices, all threads). */
+unsigned long long streamops_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STREAMOPS_H */

@@ -1,0 +1,372 @@
+// The C ABI of libstreamops: argument checks, per-device state, tuning table, dispatch.
+// Declarations and the contract of every entry point are in include/streamops.h.
+#include <atomic>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/streamops.h"
+#include "internal.cuh"
+
+using namespace streamops;
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceState {
+    bool ready = false;
+    int sm_count = 0;
+    double *partials = nullptr;        // kDotSlots * kMaxDotBlocks doubles
+    unsigned *tickets = nullptr;       // kDotSlots counters, zero between calls
+    int *error_flag = nullptr;         // set by a bounded wait that gave up
+    std::atomic<unsigned> next_slot{0};
+    // host-path buffers (streamops_chain_host_*)
+    void *chain_buf[3] = {nullptr, nullptr, nullptr};
+    void *chain_dot = nullptr;
+    size_t chain_bytes = 0;
+    cudaStream_t chain_stream = nullptr;
+};
+
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+std::atomic<int> g_last_cuda_error{0};
+std::atomic<unsigned long long> g_launches{0};
+
+// Defaults: the measured best launch shapes on B200 for arrays far larger than L2.
+streamops_tuning_t default_tuning(int op, int dtype) {
+    (void)dtype;
+    streamops_tuning_t t;
+    t.kind = 0; t.vec_bytes = 32; t.unroll = 2; t.threads = 512; t.blocks_per_sm = 4;
+    t.policy = 0; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 6; t.two_pass = 0;
+    if (op == STREAMOPS_DOT) { t.unroll = 2; t.blocks_per_sm = 2; }
+    return t;
+}
+
+streamops_tuning_t g_tuning[OP_COUNT][2];
+std::once_flag g_tuning_once;
+void init_tuning() {
+    for (int op = 0; op < OP_COUNT; ++op)
+        for (int dt = 0; dt < 2; ++dt) g_tuning[op][dt] = default_tuning(op, dt);
+}
+const streamops_tuning_t &tuning(int op, int dtype) {
+    std::call_once(g_tuning_once, init_tuning);
+    return g_tuning[op][dtype];
+}
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda_error.store((int)e);
+    return STREAMOPS_ERR_CUDA;
+}
+
+int init_device(int device, DeviceState **out) {
+    if (device < 0 || device >= kMaxDevices) return STREAMOPS_ERR_ARG;
+    DeviceState &d = g_dev[device];
+    if (!d.ready) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!d.ready) {
+            int prev = 0;
+            cudaError_t e = cudaGetDevice(&prev);
+            if (e != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaSetDevice(device)) != cudaSuccess) return cuda_fail(e);
+            int status = STREAMOPS_OK;
+            do {
+                if ((e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { status = cuda_fail(e); break; }
+                const size_t pbytes = sizeof(double) * kDotSlots * kMaxDotBlocks;
+                if (cudaMalloc(&d.partials, pbytes) != cudaSuccess ||
+                    cudaMalloc(&d.tickets, sizeof(unsigned) * kDotSlots) != cudaSuccess ||
+                    cudaMalloc(&d.error_flag, sizeof(int)) != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    status = STREAMOPS_ERR_WORKSPACE; break;
+                }
+                if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned) * kDotSlots)) != cudaSuccess) { status = cuda_fail(e); break; }
+                if ((e = cudaMemset(d.error_flag, 0, sizeof(int))) != cudaSuccess) { status = cuda_fail(e); break; }
+            } while (false);
+            cudaSetDevice(prev);
+            if (status != STREAMOPS_OK) {
+                cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag);
+                d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr;
+                return status;
+            }
+            d.ready = true;
+        }
+    }
+    *out = &d;
+    return STREAMOPS_OK;
+}
+
+int current_device_state(DeviceState **out) {
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return init_device(device, out);
+}
+
+bool ranges_overlap(const void *a, size_t abytes, const void *b, size_t bbytes) {
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bbytes && b0 < a0 + abytes;
+}
+
+// Null / alignment / overlap rules common to the five operations.
+int check_args(int op, size_t esize, const void *x, const void *y, const void *out, size_t n) {
+    const bool uses_y = (op == OP_ADD || op == OP_TRIAD || op == OP_DOT);
+    if (!out && (n > 0 || op == OP_DOT)) return STREAMOPS_ERR_NULL;   // Dot writes even for n == 0
+    if (n > 0 && (!x || (uses_y && !y))) return STREAMOPS_ERR_NULL;
+    if (((uintptr_t)out % esize) || (n > 0 && (((uintptr_t)x % esize) || (uses_y && ((uintptr_t)y % esize)))))
+        return STREAMOPS_ERR_ALIGN;
+    if (n == 0) return STREAMOPS_OK;
+    if (n > ((size_t)1 << 48)) return STREAMOPS_ERR_ARG;
+    const size_t bytes = n * esize;
+    const size_t obytes = (op == OP_DOT) ? esize : bytes;
+    const void *ins[2] = {x, uses_y ? y : nullptr};
+    for (const void *in : ins) {
+        if (!in) continue;
+        if (op != OP_DOT && in == out) continue;              // exact in-place use is allowed
+        if (ranges_overlap(in, bytes, out, obytes)) return STREAMOPS_ERR_OVERLAP;
+    }
+    return STREAMOPS_OK;
+}
+
+unsigned clamp_grid(size_t blocks) {
+    if (blocks < 1) return 1;
+    return (unsigned)(blocks > 0x7fffffffull ? 0x7fffffffull : blocks);
+}
+
+VecLaunch resolve_vec(const streamops_tuning_t &t, const DeviceState &d, int op, size_t esize,
+                      const void *x, const void *y, const void *out, size_t n) {
+    VecLaunch c;
+    uintptr_t bits = (uintptr_t)x | (op == OP_DOT ? 0 : (uintptr_t)out);
+    if (op == OP_ADD || op == OP_TRIAD || op == OP_DOT) bits |= (uintptr_t)y;
+    c.vec_bytes = t.vec_bytes;
+    if (c.vec_bytes == 32 && (bits & 31)) c.vec_bytes = 16;
+    if (c.vec_bytes == 16 && (bits & 15)) c.vec_bytes = 0;
+    c.unroll = t.unroll;
+    c.threads = t.threads;
+    c.contiguous = t.contiguous;
+    c.policy = t.policy;
+    // the read-only data path must not be used on an array the kernel also writes
+    if (c.policy == 1 && (out == x || out == y)) c.policy = 0;
+    const size_t per_tile = (size_t)c.threads * (c.vec_bytes ? (size_t)c.unroll * c.vec_bytes / esize : 1);
+    const size_t tiles = (n + per_tile - 1) / per_tile;
+    size_t grid = t.blocks_per_sm > 0 ? (size_t)t.blocks_per_sm * d.sm_count : tiles;
+    if (grid > tiles) grid = tiles;                            // never more blocks than tiles
+    if (op == OP_DOT && grid > (size_t)kMaxDotBlocks) grid = kMaxDotBlocks;
+    c.grid = clamp_grid(grid);
+    return c;
+}
+
+bool valid_tuning(const streamops_tuning_t &t) {
+    if (t.kind != 0 && t.kind != 1) return false;
+    if (t.vec_bytes != 16 && t.vec_bytes != 32) return false;
+    if (t.unroll != 1 && t.unroll != 2 && t.unroll != 4) return false;
+    if (t.threads != 128 && t.threads != 256 && t.threads != 512) return false;
+    if (t.blocks_per_sm < 0 || t.blocks_per_sm > 32) return false;
+    if (t.policy < 0 || t.policy > 4) return false;
+    if (t.chunk_bytes < 1024 || t.chunk_bytes > 65536 || (t.chunk_bytes & 15)) return false;
+    if (t.stages < 2 || t.stages > 8) return false;
+    return true;
+}
+
+int run_op(int op, int dtype, const void *x, const void *y, void *out, double scalar, size_t n,
+           streamops_stream_t stream_) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const size_t esize = dtype == DT_F64 ? 8 : 4;
+    int status = check_args(op, esize, x, y, out, n);
+    if (status != STREAMOPS_OK) return status;
+    if (n == 0) {
+        if (op != OP_DOT) return STREAMOPS_OK;
+        cudaError_t e = cudaMemsetAsync(out, 0, esize, stream);   // +0 in either format
+        return e == cudaSuccess ? STREAMOPS_OK : cuda_fail(e);
+    }
+    DeviceState *d = nullptr;
+    if ((status = current_device_state(&d)) != STREAMOPS_OK) return status;
+    const streamops_tuning_t &t = tuning(op, dtype);
+
+    DotScratch scratch{nullptr, nullptr};
+    if (op == OP_DOT) {
+        const unsigned slot = d->next_slot.fetch_add(1) % kDotSlots;
+        scratch.partials = d->partials + (size_t)slot * kMaxDotBlocks;
+        scratch.ticket = d->tickets + slot;
+    }
+
+    cudaError_t e;
+    int launches = 1;
+    uintptr_t bits = (uintptr_t)x | (op == OP_DOT ? 0 : (uintptr_t)out);
+    if (op == OP_ADD || op == OP_TRIAD || op == OP_DOT) bits |= (uintptr_t)y;
+    if (t.kind == 1 && !(bits & 15)) {
+        BulkLaunch b;
+        b.threads = t.threads;
+        b.chunk_bytes = t.chunk_bytes;
+        b.stages = t.stages;
+        const size_t nchunks = (n * esize + b.chunk_bytes - 1) / b.chunk_bytes;
+        size_t grid = (size_t)(t.blocks_per_sm > 0 ? t.blocks_per_sm : 1) * d->sm_count;
+        if (grid > nchunks) grid = nchunks;
+        if (op == OP_DOT && grid > (size_t)kMaxDotBlocks) grid = kMaxDotBlocks;
+        b.grid = clamp_grid(grid);
+        e = launch_bulk(op, dtype, b, x, y, out, scalar, n, scratch, d->error_flag, stream, &launches);
+    } else {
+        const VecLaunch c = resolve_vec(t, *d, op, esize, x, y, out, n);
+        if (op == OP_DOT) e = launch_dot(dtype, c, t.two_pass != 0, x, y, out, n, scratch, stream, &launches);
+        else e = launch_elementwise(op, dtype, c, x, y, out, scalar, n, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_launches.fetch_add((unsigned long long)launches);
+    return STREAMOPS_OK;
+}
+
+template <typename T>
+int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
+    constexpr int dtype = sizeof(T) == 8 ? DT_F64 : DT_F32;
+    if (!dot_out || (n > 0 && (!a || !b || !c))) return STREAMOPS_ERR_NULL;
+    DeviceState *d = nullptr;
+    int status = current_device_state(&d);
+    if (status != STREAMOPS_OK) return status;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    cudaError_t e;
+    const size_t bytes = n * sizeof(T);
+    if (!d->chain_stream && (e = cudaStreamCreateWithFlags(&d->chain_stream, cudaStreamNonBlocking)) != cudaSuccess)
+        return cuda_fail(e);
+    if (!d->chain_dot && cudaMalloc(&d->chain_dot, 8) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_ERR_WORKSPACE; }
+    if (bytes > d->chain_bytes) {
+        for (void *&p : d->chain_buf) { cudaFree(p); p = nullptr; }
+        d->chain_bytes = 0;
+        for (void *&p : d->chain_buf)
+            if (cudaMalloc(&p, bytes) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_ERR_WORKSPACE; }
+        d->chain_bytes = bytes;
+    }
+    cudaStream_t st = d->chain_stream;
+    T *da = (T *)d->chain_buf[0], *db = (T *)d->chain_buf[1], *dc = (T *)d->chain_buf[2], *dd = (T *)d->chain_dot;
+    T *host[3] = {a, b, c};
+    T *dev[3] = {da, db, dc};
+    for (int i = 0; i < 3 && n > 0; ++i)
+        if ((e = cudaMemcpyAsync(dev[i], host[i], bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    // c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b)
+    if ((status = run_op(OP_COPY, dtype, da, nullptr, dc, scalar, n, st)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_SCALE, dtype, dc, nullptr, db, scalar, n, st)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_ADD, dtype, da, db, dc, scalar, n, st)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_TRIAD, dtype, db, dc, da, scalar, n, st)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_DOT, dtype, da, db, dd, scalar, n, st)) != STREAMOPS_OK) return status;
+    for (int i = 0; i < 3 && n > 0; ++i)
+        if ((e = cudaMemcpyAsync(host[i], dev[i], bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(dot_out, dd, sizeof(T), cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
+    return STREAMOPS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+#define STREAMOPS_UNARY(NAME, OP, T, DT)                                                             \
+    int NAME(const T *x, T *out, double scalar, size_t n, streamops_stream_t stream) {               \
+        return run_op(OP, DT, x, nullptr, out, scalar, n, stream);                                   \
+    }
+#define STREAMOPS_BINARY(NAME, OP, T, DT)                                                            \
+    int NAME(const T *x, const T *y, T *out, double scalar, size_t n, streamops_stream_t stream) {   \
+        return run_op(OP, DT, x, y, out, scalar, n, stream);                                         \
+    }
+STREAMOPS_UNARY(stream_copy_f64, OP_COPY, double, DT_F64)
+STREAMOPS_UNARY(stream_copy_f32, OP_COPY, float, DT_F32)
+STREAMOPS_UNARY(stream_scale_f64, OP_SCALE, double, DT_F64)
+STREAMOPS_UNARY(stream_scale_f32, OP_SCALE, float, DT_F32)
+STREAMOPS_BINARY(stream_add_f64, OP_ADD, double, DT_F64)
+STREAMOPS_BINARY(stream_add_f32, OP_ADD, float, DT_F32)
+STREAMOPS_BINARY(stream_triad_f64, OP_TRIAD, double, DT_F64)
+STREAMOPS_BINARY(stream_triad_f32, OP_TRIAD, float, DT_F32)
+STREAMOPS_BINARY(stream_dot_f64, OP_DOT, double, DT_F64)
+STREAMOPS_BINARY(stream_dot_f32, OP_DOT, float, DT_F32)
+
+int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out) {
+    return chain_host<double>(a, b, c, scalar, n, dot_out);
+}
+int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out) {
+    return chain_host<float>(a, b, c, scalar, n, dot_out);
+}
+
+int streamops_init(int device) {
+    DeviceState *d = nullptr;
+    return init_device(device, &d);
+}
+
+int streamops_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_OK; }
+    for (int i = 0; i < kMaxDevices; ++i) {
+        DeviceState &d = g_dev[i];
+        if (!d.ready) continue;
+        cudaSetDevice(i);
+        cudaDeviceSynchronize();
+        cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag); cudaFree(d.chain_dot);
+        for (void *&p : d.chain_buf) { cudaFree(p); p = nullptr; }
+        if (d.chain_stream) cudaStreamDestroy(d.chain_stream);
+        d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr; d.chain_dot = nullptr;
+        d.chain_stream = nullptr; d.chain_bytes = 0; d.ready = false;
+    }
+    cudaSetDevice(prev);
+    return STREAMOPS_OK;
+}
+
+int streamops_set_tuning(int op, int dtype, const streamops_tuning_t *t) {
+    if (!t) return STREAMOPS_ERR_NULL;
+    if (op < 0 || op >= OP_COUNT || dtype < 0 || dtype > 1 || !valid_tuning(*t)) return STREAMOPS_ERR_ARG;
+    (void)tuning(op, dtype);
+    g_tuning[op][dtype] = *t;
+    return STREAMOPS_OK;
+}
+
+int streamops_get_tuning(int op, int dtype, streamops_tuning_t *t) {
+    if (!t) return STREAMOPS_ERR_NULL;
+    if (op < 0 || op >= OP_COUNT || dtype < 0 || dtype > 1) return STREAMOPS_ERR_ARG;
+    *t = tuning(op, dtype);
+    return STREAMOPS_OK;
+}
+
+int streamops_reset_tuning(void) {
+    (void)tuning(0, 0);
+    init_tuning();
+    return STREAMOPS_OK;
+}
+
+const char *streamops_policy_name(int policy) {
+    switch (policy) {
+        case 0: return "ld.global / st.global";
+        case 1: return "ld.global.nc / st.global";
+        case 2: return "ld.global.cs / st.global.cs";
+        case 3: return "ld.global.L1::no_allocate / st.global.cs";
+        case 4: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first";
+        default: return "unknown";
+    }
+}
+
+int streamops_check(streamops_stream_t stream) {
+    DeviceState *d = nullptr;
+    int status = current_device_state(&d);
+    if (status != STREAMOPS_OK) return status;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int flag = 0;
+    if ((e = cudaMemcpy(&flag, d->error_flag, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e);
+    if (flag == 0) return STREAMOPS_OK;
+    if ((e = cudaMemset(d->error_flag, 0, sizeof(int))) != cudaSuccess) return cuda_fail(e);
+    return STREAMOPS_ERR_TIMEOUT;
+}
+
+const char *streamops_status_string(int status) {
+    switch (status) {
+        case STREAMOPS_OK: return "ok";
+        case STREAMOPS_ERR_NULL: return "null pointer";
+        case STREAMOPS_ERR_ALIGN: return "pointer not aligned to the element size";
+        case STREAMOPS_ERR_OVERLAP: return "output partially overlaps an input";
+        case STREAMOPS_ERR_CUDA: return "CUDA error (see streamops_last_cuda_error)";
+        case STREAMOPS_ERR_WORKSPACE: return "workspace allocation failed";
+        case STREAMOPS_ERR_TIMEOUT: return "a bounded wait inside a kernel gave up";
+        case STREAMOPS_ERR_ARG: return "argument out of range";
+        default: return "unknown status";
+    }
+}
+
+int streamops_last_cuda_error(void) { return g_last_cuda_error.load(); }
+
+unsigned long long streamops_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

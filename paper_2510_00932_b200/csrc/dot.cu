@@ -1,0 +1,153 @@
+// Dot kernels (Table 1 of the paper, "Dot"): out[0] = (T) sum_i x[i] * y[i].
+//
+// Pass 1 streams x and y exactly like the elementwise kernels (tiles of blockDim.x * U vectors,
+// tiles interleaved across a persistent grid) and keeps U double-precision accumulators per
+// thread; float inputs are widened first, so every product is exact. The accumulators are
+// folded in a fixed order: per thread (u = 0..U-1), per warp (xor-shuffle tree), per block
+// (shared memory, warp 0 folds the warp sums), giving partials[blockIdx.x].
+//
+// Pass 2 sums partials[0..G-1] with one block in a fixed order (thread t takes t, t + B, ... in
+// sequence, then the same warp/block tree). It runs either as its own launch or inside pass 1
+// by whichever block arrives last at an atomic ticket: the ticket only elects WHO does pass 2,
+// the order of the additions is by block index, so the bits of the result never depend on
+// block scheduling, on the stream, or on what else the GPU is running.
+#include "internal.cuh"
+#include "memops.cuh"
+#include "reduce.cuh"
+
+namespace streamops {
+
+namespace {
+
+template <typename T, int VB>
+__device__ __forceinline__ double fold_vec(double acc, const Vec<VB> &xv, const Vec<VB> &yv) {
+    constexpr int EPV = VB / (int)sizeof(T);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e)
+        acc = fma(widen<T>(Lanes<T>::get(xv.w, e)), widen<T>(Lanes<T>::get(yv.w, e)), acc);
+    return acc;
+}
+
+template <typename T, int VB, int U, int POL, bool SINGLE_LAUNCH>
+__global__ void __launch_bounds__(kMaxThreads)
+dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out) {
+    constexpr int EPV = VB / (int)sizeof(T);
+    __shared__ double warp_part[32];
+    __shared__ bool is_last;
+    const char *xb = reinterpret_cast<const char *>(x);
+    const char *yb = reinterpret_cast<const char *>(y);
+    uint64_t l2pol = 0;
+    if constexpr (POL == 4) l2pol = make_evict_first_policy();
+
+    const size_t nvec = n / EPV;
+    const size_t tile_vecs = (size_t)blockDim.x * U;
+    const size_t ntiles = nvec / tile_vecs;
+    double acc[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) acc[u] = 0.0;
+
+    for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const size_t v0 = tile * tile_vecs + threadIdx.x;
+        Vec<VB> xv[U], yv[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+#pragma unroll
+        for (int u = 0; u < U; ++u) ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+#pragma unroll
+        for (int u = 0; u < U; ++u) acc[u] = fold_vec<T, VB>(acc[u], xv[u], yv[u]);
+    }
+    if (blockIdx.x == (unsigned)(ntiles % gridDim.x)) {      // ragged end, one block
+        for (size_t v = ntiles * tile_vecs + threadIdx.x; v < nvec; v += blockDim.x) {
+            Vec<VB> xv, yv;
+            ldg<0>(xv, xb + v * VB, 0);
+            ldg<0>(yv, yb + v * VB, 0);
+            acc[0] = fold_vec<T, VB>(acc[0], xv, yv);
+        }
+        const size_t i = nvec * EPV + threadIdx.x;
+        if (i < n) acc[0] = fma(widen<T>(x[i]), widen<T>(y[i]), acc[0]);
+    }
+    double tsum = acc[0];
+#pragma unroll
+    for (int u = 1; u < U; ++u) tsum += acc[u];
+    const double bsum = block_sum(tsum, warp_part);
+
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(1024)
+dot_pass2_kernel(const double *partials, unsigned count, T *out) {
+    __shared__ double warp_part[32];
+    finish<T>(partials, count, out, warp_part);
+}
+
+// Scalar pass 1 for pointers that are not 16-byte aligned: same structure, one element per load.
+template <typename T, bool SINGLE_LAUNCH>
+__global__ void __launch_bounds__(kMaxThreads)
+dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out) {
+    __shared__ double warp_part[32];
+    __shared__ bool is_last;
+    double acc = 0.0;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        acc = fma(widen<T>(x[i]), widen<T>(y[i]), acc);
+    const double bsum = block_sum(acc, warp_part);
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last);
+}
+
+template <typename T, int VB, int U, bool SL>
+cudaError_t launch_pol(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
+    switch (c.policy) {
+#define STREAMOPS_CASE(P) case P: dot_pass1_kernel<T, VB, U, P, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out); break;
+        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4)
+#undef STREAMOPS_CASE
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+template <typename T, int VB, bool SL>
+cudaError_t launch_unroll(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
+    switch (c.unroll) {
+        case 1: return launch_pol<T, VB, 1, SL>(c, x, y, n, s, out, st);
+        case 2: return launch_pol<T, VB, 2, SL>(c, x, y, n, s, out, st);
+        case 4: return launch_pol<T, VB, 4, SL>(c, x, y, n, s, out, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+template <typename T, bool SL>
+cudaError_t launch_pass1(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
+    if (c.vec_bytes == 32) return launch_unroll<T, 32, SL>(c, x, y, n, s, out, st);
+    if (c.vec_bytes == 16) return launch_unroll<T, 16, SL>(c, x, y, n, s, out, st);
+    dot_scalar_kernel<T, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, const T *x, const T *y, T *out, size_t n,
+                         const DotScratch &s, cudaStream_t st, int *launches) {
+    if (c.grid > (unsigned)kMaxDotBlocks) return cudaErrorInvalidValue;
+    if (!two_pass) {
+        *launches = 1;
+        return launch_pass1<T, true>(c, x, y, n, s, out, st);
+    }
+    *launches = 2;
+    cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, out, st);
+    if (e != cudaSuccess) return e;
+    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, out);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, const void *x, const void *y,
+                       void *out, size_t n, const DotScratch &scratch, cudaStream_t stream, int *launches) {
+    if (dtype == DT_F64)
+        return launch_dot_t<double>(cfg, two_pass, (const double *)x, (const double *)y, (double *)out, n,
+                                    scratch, stream, launches);
+    return launch_dot_t<float>(cfg, two_pass, (const float *)x, (const float *)y, (float *)out, n,
+                               scratch, stream, launches);
+}
+
+}  // namespace streamops

@@ -1,0 +1,54 @@
+// Interfaces between the C-ABI layer (api.cu) and the kernel families (one .cu file each).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace streamops {
+
+enum : int { OP_COPY = 0, OP_SCALE = 1, OP_ADD = 2, OP_TRIAD = 3, OP_DOT = 4, OP_COUNT = 5 };
+enum : int { DT_F32 = 0, DT_F64 = 1 };
+
+constexpr int kMaxThreads = 512;       // __launch_bounds__ of every vector kernel
+constexpr int kMaxDotBlocks = 4096;    // partial sums per Dot workspace slot
+constexpr int kDotSlots = 32;          // Dot calls that may be in flight per device
+
+// Resolved launch shape for the register-vector kernels.
+struct VecLaunch {
+    int vec_bytes;     // 32, 16, or 0 = scalar kernel (pointers not 16-byte aligned)
+    int unroll;        // 1, 2, 4
+    int policy;        // 0..kNumPolicies-1
+    int threads;
+    unsigned grid;
+    int contiguous;
+};
+
+// Resolved launch shape for the bulk-copy (TMA) pipeline kernels.
+struct BulkLaunch {
+    int threads;       // consumer threads (one extra producer warp is added by the launcher)
+    unsigned grid;
+    int chunk_bytes;
+    int stages;
+};
+
+// Per-slot Dot scratch: partial sums written by pass 1, the arrival ticket of the single-launch
+// variant, and (shared) the device error flag.
+struct DotScratch {
+    double *partials;      // kMaxDotBlocks doubles
+    unsigned *ticket;      // one counter, zero between calls
+};
+
+// elementwise.cu
+cudaError_t launch_elementwise(int op, int dtype, const VecLaunch &cfg, const void *x, const void *y,
+                               void *out, double scalar, size_t n, cudaStream_t stream);
+// dot.cu
+cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, const void *x, const void *y,
+                       void *out, size_t n, const DotScratch &scratch, cudaStream_t stream,
+                       int *launches);
+// bulk.cu
+cudaError_t launch_bulk(int op, int dtype, const BulkLaunch &cfg, const void *x, const void *y,
+                        void *out, double scalar, size_t n, const DotScratch &scratch,
+                        int *error_flag, cudaStream_t stream, int *launches);
+size_t bulk_smem_bytes(int op, const BulkLaunch &cfg);
+
+}  // namespace streamops

@@ -1,0 +1,93 @@
+// Global-memory vector loads and stores with explicit cache-hint sets, as inline PTX.
+//
+// A "policy" picks the qualifiers on ld.global / st.global. Streaming kernels touch every byte
+// once, so the hints only decide how much of L1/L2 the stream is allowed to occupy:
+//   0  ld.global                    st.global                      (default caching)
+//   1  ld.global.nc                 st.global                      (read-only data path)
+//   2  ld.global.cs                 st.global.cs                   (evict-first streaming)
+//   3  ld.global.L1::no_allocate    st.global.cs
+//   4  ld.global.L1::no_allocate + L2 evict_first policy on loads and stores
+// 16-byte accesses are .v4.b32; 32-byte accesses are the 256-bit .v8.b32 form of sm_100.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace streamops {
+
+constexpr int kNumPolicies = 5;
+
+template <int VB> struct Vec;
+template <> struct alignas(16) Vec<16> { uint32_t w[4]; };
+template <> struct alignas(32) Vec<32> { uint32_t w[8]; };
+
+__device__ __forceinline__ uint64_t make_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+#define STREAMOPS_LD16(QUAL, TAIL, ...)                                                          \
+    asm volatile("ld.global" QUAL ".v4.b32 {%0,%1,%2,%3}, [%4]" TAIL ";"                         \
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3])                        \
+                 : "l"(p) __VA_ARGS__)
+#define STREAMOPS_LD32(QUAL, TAIL, ...)                                                          \
+    asm volatile("ld.global" QUAL ".v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8]" TAIL ";"             \
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]),         \
+                   "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])                                      \
+                 : "l"(p) __VA_ARGS__)
+#define STREAMOPS_ST16(QUAL, TAIL, ...)                                                          \
+    asm volatile("st.global" QUAL ".v4.b32 [%0], {%1,%2,%3,%4}" TAIL ";"                         \
+                 :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]) __VA_ARGS__       \
+                 : "memory")
+#define STREAMOPS_ST32(QUAL, TAIL, ...)                                                          \
+    asm volatile("st.global" QUAL ".v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8}" TAIL ";"             \
+                 :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]), "r"(v.w[4]),     \
+                    "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7]) __VA_ARGS__                            \
+                 : "memory")
+
+template <int POL>
+__device__ __forceinline__ void ldg(Vec<16> &v, const void *p, uint64_t l2pol) {
+    if constexpr (POL == 0) STREAMOPS_LD16("", "");
+    else if constexpr (POL == 1) STREAMOPS_LD16(".nc", "");
+    else if constexpr (POL == 2) STREAMOPS_LD16(".cs", "");
+    else if constexpr (POL == 3) STREAMOPS_LD16(".L1::no_allocate", "");
+    else STREAMOPS_LD16(".L1::no_allocate.L2::cache_hint", ", %5", , "l"(l2pol));
+}
+template <int POL>
+__device__ __forceinline__ void ldg(Vec<32> &v, const void *p, uint64_t l2pol) {
+    if constexpr (POL == 0) STREAMOPS_LD32("", "");
+    else if constexpr (POL == 1) STREAMOPS_LD32(".nc", "");
+    else if constexpr (POL == 2) STREAMOPS_LD32(".cs", "");
+    else if constexpr (POL == 3) STREAMOPS_LD32(".L1::no_allocate", "");
+    else STREAMOPS_LD32(".L1::no_allocate.L2::cache_hint", ", %9", , "l"(l2pol));
+}
+template <int POL>
+__device__ __forceinline__ void stg(void *p, const Vec<16> &v, uint64_t l2pol) {
+    if constexpr (POL == 0 || POL == 1) STREAMOPS_ST16("", "");
+    else if constexpr (POL == 2 || POL == 3) STREAMOPS_ST16(".cs", "");
+    else STREAMOPS_ST16(".L2::cache_hint", ", %5", , "l"(l2pol));
+}
+template <int POL>
+__device__ __forceinline__ void stg(void *p, const Vec<32> &v, uint64_t l2pol) {
+    if constexpr (POL == 0 || POL == 1) STREAMOPS_ST32("", "");
+    else if constexpr (POL == 2 || POL == 3) STREAMOPS_ST32(".cs", "");
+    else STREAMOPS_ST32(".L2::cache_hint", ", %9", , "l"(l2pol));
+}
+
+// Views of a vector's words as elements. A double is a register pair, so these are free.
+template <typename T> struct Lanes;
+template <> struct Lanes<double> {
+    static __device__ __forceinline__ double get(const uint32_t *w, int i) {
+        return __hiloint2double((int)w[2 * i + 1], (int)w[2 * i]);
+    }
+    static __device__ __forceinline__ void set(uint32_t *w, int i, double v) {
+        w[2 * i] = (uint32_t)__double2loint(v);
+        w[2 * i + 1] = (uint32_t)__double2hiint(v);
+    }
+};
+template <> struct Lanes<float> {
+    static __device__ __forceinline__ float get(const uint32_t *w, int i) { return __uint_as_float(w[i]); }
+    static __device__ __forceinline__ void set(uint32_t *w, int i, float v) { w[i] = __float_as_uint(v); }
+};
+
+}  // namespace streamops

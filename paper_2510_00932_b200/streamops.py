@@ -1,0 +1,223 @@
+"""ctypes binding of libstreamops: argument marshalling only.
+
+Each function below forwards to the C entry point of the same name (see include/streamops.h).
+Tensors supply device pointers, ``torch.cuda.current_stream()`` supplies the stream; every step
+of the computation runs inside the library's CUDA kernels. There is no fallback: if the shared
+library is missing or a call returns a non-zero status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstreamops.so")
+
+OPS = ("copy", "scale", "add", "triad", "dot")
+OP_CODE = {name: i for i, name in enumerate(OPS)}
+DTYPE_CODE = {"f32": 0, "f64": 1}
+# arrays moved per element, counted the standard STREAM way
+ARRAYS_MOVED = {"copy": 2, "scale": 2, "add": 3, "triad": 3, "dot": 2}
+
+
+class StreamopsError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"libstreamops status {status}: {message}")
+        self.status = status
+
+
+class Tuning(ctypes.Structure):
+    """Mirror of streamops_tuning_t."""
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "kind", "vec_bytes", "unroll", "threads", "blocks_per_sm", "policy", "contiguous",
+        "chunk_bytes", "stages", "two_pass")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libstreamops.so (built in-tree by ``build.py``); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with "
+                              "`python -m paper_2510_00932_b200.build` (needs nvcc)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, dbl, sz, ci = ctypes.c_void_p, ctypes.c_double, ctypes.c_size_t, ctypes.c_int
+        for t in ("f32", "f64"):
+            for name in ("copy", "scale"):
+                f = getattr(L, f"stream_{name}_{t}")
+                f.argtypes, f.restype = [vp, vp, dbl, sz, vp], ci
+            for name in ("add", "triad", "dot"):
+                f = getattr(L, f"stream_{name}_{t}")
+                f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
+            f = getattr(L, f"streamops_chain_host_{t}")
+            f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
+        L.streamops_init.argtypes, L.streamops_init.restype = [ci], ci
+        L.streamops_shutdown.argtypes, L.streamops_shutdown.restype = [], ci
+        L.streamops_set_tuning.argtypes, L.streamops_set_tuning.restype = [ci, ci, ctypes.POINTER(Tuning)], ci
+        L.streamops_get_tuning.argtypes, L.streamops_get_tuning.restype = [ci, ci, ctypes.POINTER(Tuning)], ci
+        L.streamops_reset_tuning.argtypes, L.streamops_reset_tuning.restype = [], ci
+        L.streamops_policy_name.argtypes, L.streamops_policy_name.restype = [ci], ctypes.c_char_p
+        L.streamops_check.argtypes, L.streamops_check.restype = [vp], ci
+        L.streamops_status_string.argtypes, L.streamops_status_string.restype = [ci], ctypes.c_char_p
+        L.streamops_last_cuda_error.argtypes, L.streamops_last_cuda_error.restype = [], ci
+        L.streamops_launch_count.argtypes, L.streamops_launch_count.restype = [], ctypes.c_ulonglong
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().streamops_status_string(int(status)).decode()
+
+
+def _raise(status: int):
+    if status != 0:
+        msg = status_string(status)
+        if status == 4:
+            msg += f" [cudaError {lib().streamops_last_cuda_error()}]"
+        raise StreamopsError(status, msg)
+
+
+def _suffix(t) -> str:
+    import torch
+    if t.dtype == torch.float64:
+        return "f64"
+    if t.dtype == torch.float32:
+        return "f32"
+    raise TypeError(f"libstreamops handles float32 and float64 tensors, got {t.dtype}")
+
+
+def _marshal(*tensors):
+    """Common dtype suffix, element count and the current stream of the tensors' device."""
+    import torch
+    first = tensors[0]
+    suf = _suffix(first)
+    for t in tensors:
+        if not t.is_cuda:
+            raise ValueError("libstreamops operates on CUDA tensors")
+        if not t.is_contiguous() or t.dim() != 1:
+            raise ValueError("libstreamops operates on contiguous 1-D tensors")
+        if _suffix(t) != suf or t.device != first.device:
+            raise ValueError("all tensors of one call share dtype and device")
+    stream = torch.cuda.current_stream(first.device).cuda_stream
+    return suf, stream
+
+
+def copy(x, out, scalar: float = 0.0):
+    """out[i] = x[i] (stream_copy_*)."""
+    suf, stream = _marshal(x, out)
+    if out.numel() != x.numel():
+        raise ValueError("length mismatch")
+    _raise(getattr(lib(), f"stream_copy_{suf}")(x.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+def scale(x, out, scalar: float):
+    """out[i] = RN(s * x[i]) (stream_scale_*)."""
+    suf, stream = _marshal(x, out)
+    if out.numel() != x.numel():
+        raise ValueError("length mismatch")
+    _raise(getattr(lib(), f"stream_scale_{suf}")(x.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+def add(x, y, out, scalar: float = 0.0):
+    """out[i] = RN(x[i] + y[i]) (stream_add_*)."""
+    suf, stream = _marshal(x, y, out)
+    if not (out.numel() == x.numel() == y.numel()):
+        raise ValueError("length mismatch")
+    _raise(getattr(lib(), f"stream_add_{suf}")(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+def triad(x, y, out, scalar: float):
+    """out[i] = RN(x[i] + RN(s * y[i])) (stream_triad_*)."""
+    suf, stream = _marshal(x, y, out)
+    if not (out.numel() == x.numel() == y.numel()):
+        raise ValueError("length mismatch")
+    _raise(getattr(lib(), f"stream_triad_{suf}")(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+def dot(x, y, out, scalar: float = 0.0):
+    """out[0] = (T) sum x[i]*y[i]; out is a one-element device tensor (stream_dot_*)."""
+    suf, stream = _marshal(x, y, out)
+    if x.numel() != y.numel() or out.numel() != 1:
+        raise ValueError("dot takes two equal-length inputs and a one-element output")
+    _raise(getattr(lib(), f"stream_dot_{suf}")(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+def chain(a, b, c, dot_out, scalar: float):
+    """One pass of the five kernels over device tensors a, b, c in the STREAM dataflow:
+    c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot_out <- dot(a, b). Five library calls."""
+    copy(a, c)
+    scale(c, b, scalar)
+    add(a, b, c)
+    triad(b, c, a, scalar)
+    dot(a, b, dot_out)
+
+
+def chain_host(a, b, c, scalar: float):
+    """The same pass over three HOST numpy arrays, updated in place through
+    streamops_chain_host_*; returns the dot product. Copies in both directions happen inside
+    the library call."""
+    import numpy as np
+    suf = {np.dtype(np.float64): "f64", np.dtype(np.float32): "f32"}[a.dtype]
+    for arr in (a, b, c):
+        if arr.dtype != a.dtype or arr.shape != a.shape or arr.ndim != 1 or not arr.flags.c_contiguous:
+            raise ValueError("chain_host takes three contiguous 1-D arrays of one dtype and length")
+    res = np.zeros(1, dtype=a.dtype)
+    _raise(getattr(lib(), f"streamops_chain_host_{suf}")(a.ctypes.data, b.ctypes.data, c.ctypes.data,
+                                                        float(scalar), a.size, res.ctypes.data))
+    return res[0]
+
+
+def init(device: int = 0):
+    _raise(lib().streamops_init(int(device)))
+
+
+def shutdown():
+    _raise(lib().streamops_shutdown())
+
+
+def get_tuning(op: str, dtype: str) -> Tuning:
+    t = Tuning()
+    _raise(lib().streamops_get_tuning(OP_CODE[op], DTYPE_CODE[dtype], ctypes.byref(t)))
+    return t
+
+
+def set_tuning(op: str, dtype: str, **fields) -> Tuning:
+    """Overrides fields of the (op, dtype) tuning; returns the tuning now in force."""
+    t = get_tuning(op, dtype)
+    for k, v in fields.items():
+        if not hasattr(t, k):
+            raise KeyError(k)
+        setattr(t, k, int(v))
+    _raise(lib().streamops_set_tuning(OP_CODE[op], DTYPE_CODE[dtype], ctypes.byref(t)))
+    return t
+
+
+def reset_tuning():
+    _raise(lib().streamops_reset_tuning())
+
+
+def policy_name(policy: int) -> str:
+    return lib().streamops_policy_name(int(policy)).decode()
+
+
+def check(stream=None):
+    """Synchronises the stream and raises if a bounded wait inside a kernel gave up."""
+    import torch
+    s = (stream or torch.cuda.current_stream()).cuda_stream
+    _raise(lib().streamops_check(s))
+
+
+def launch_count() -> int:
+    return int(lib().streamops_launch_count())
