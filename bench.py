@@ -30,7 +30,13 @@ UNIT = "GB/s"
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # an ncu capture, keyed by (workload, op, tuning signature); absent = not captured for this build.
-NCU_TRAFFIC_BYTES: dict = {}
+NCU_TRAFFIC_BYTES: dict = {
+    # profiles/ncu_full_five_kernels_c2_fp64.md: triad read 536.887 MB + write 229.862 MB (cold L2)
+    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "policy": 4, '
+                    '"stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 766_748_928,
+    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "policy": 4, '
+                  '"stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 769_038_080,
+}
 
 
 def parse_args():
@@ -210,6 +216,22 @@ def run_ours(args):
     value, max_ms = harness.whole_job_gbs(harness.step_bytes(n, itemsize) * K, elapsed_ms, device)
     ms_per_step = max_ms / K
 
+    # second timed region, op-major: each kernel K times back to back, so that every launch pays
+    # for its own write-backs and none inherits cached or dirty lines from a different kernel
+    iso_ms = {}
+    for name, f in calls:
+        for _ in range(3):
+            f()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(device)
+        e0.record(stream)
+        for _ in range(K):
+            f()
+        e1.record(stream)
+        torch.cuda.synchronize(device)
+        iso_ms[name] = harness.max_over_ranks(e0.elapsed_time(e1) / K, device)
+    launches = so.launch_count() - launches0
+
     # end to end: host buffers in, host buffers out, through the library's host entry point
     ha, hb, hc = (p.numpy() for p in pinned)
     e2e_steps = max(1, args.e2e_steps)
@@ -226,12 +248,14 @@ def run_ours(args):
     per_op = harness.per_op_report(op_ms, n, itemsize, peak)
     for name in per_op:
         per_op[name]["best_gbs"] = round(harness.op_bytes(name, n, itemsize) / (op_ms_best[name] * 1e-3) / 1e9, 1)
+    per_op_isolated = harness.per_op_report(iso_ms, n, itemsize, peak)
     dominant = max(op_ms, key=lambda k: op_ms[k])
     sig = tuning_signature(so, w.dtype)
     traffic = NCU_TRAFFIC_BYTES.get((w.name, dominant, json.dumps(sig[dominant], sort_keys=True)))
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": per_op[dominant]["gbs"], "peak": peak,
                 "peak_source": f"of {peak_src}", "unit": "GB/s",
-                "frac": round(per_op[dominant]["gbs"] / peak, 4), "traffic": traffic}
+                "frac": round(per_op[dominant]["gbs"] / peak, 4), "traffic": traffic,
+                "region": "chain-order steps; per_op_isolated has the same kernels timed op-major"}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and args.cpu_seconds > 0:
@@ -248,7 +272,7 @@ def run_ours(args):
             "config": {"workload": w.name, "n": n, "dist": w.dist, "seed": w.seed, "scalar": w.scalar,
                        "arrays": 3, "array_bytes": n * itemsize, "order": "chain (copy, scale, add, triad, dot per step)",
                        "l2": "no flush: each array is larger than the 126 MB L2", "parallelism": f"replicas x{world}"},
-            "clocks": clocks, "per_op": per_op, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "clocks": clocks, "per_op": per_op, "per_op_isolated": per_op_isolated, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": 3 * n * itemsize,
                     "d2h_bytes_per_step": 3 * n * itemsize + itemsize, "steps": e2e_steps},
             "gpu_launches": int(launches), "frac_nominal_8tbs": round(value / world / harness.NOMINAL_HBM_GBS, 4),

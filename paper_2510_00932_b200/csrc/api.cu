@@ -32,13 +32,21 @@ std::mutex g_mutex;
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<unsigned long long> g_launches{0};
 
-// Defaults: the measured best launch shapes on B200 for arrays far larger than L2.
+// Defaults: the measured best launch shapes on B200 for arrays far larger than L2 (fp64 n = 2^25,
+// fp32 n = 2^26). The elementwise kernels run one block per tile: the hardware block scheduler
+// then balances the two dies' unequal distance to memory better than a static persistent grid.
 streamops_tuning_t default_tuning(int op, int dtype) {
-    (void)dtype;
     streamops_tuning_t t;
-    t.kind = 0; t.vec_bytes = 32; t.unroll = 2; t.threads = 512; t.blocks_per_sm = 4;
-    t.policy = 0; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 6; t.two_pass = 0;
-    if (op == STREAMOPS_DOT) { t.unroll = 2; t.blocks_per_sm = 2; }
+    t.kind = 0; t.vec_bytes = 32; t.unroll = 2; t.threads = 256; t.blocks_per_sm = 0;
+    t.policy = 0; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0;
+    const bool f64 = dtype == DT_F64;
+    switch (op) {
+        case OP_COPY:  t.unroll = 4; break;
+        case OP_SCALE: if (f64) { t.policy = 4; } else { t.unroll = 4; t.policy = 2; } break;
+        case OP_ADD:   t.threads = 128; if (f64) { t.policy = 4; } else { t.unroll = 4; } break;
+        case OP_TRIAD: t.threads = 128; t.policy = 4; break;
+        case OP_DOT:   t.threads = 512; t.blocks_per_sm = 2; if (f64) { t.unroll = 4; } else { t.unroll = 1; t.policy = 2; } break;
+    }
     return t;
 }
 

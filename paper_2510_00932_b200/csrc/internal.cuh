@@ -10,7 +10,7 @@ enum : int { OP_COPY = 0, OP_SCALE = 1, OP_ADD = 2, OP_TRIAD = 3, OP_DOT = 4, OP
 enum : int { DT_F32 = 0, DT_F64 = 1 };
 
 constexpr int kMaxThreads = 512;       // __launch_bounds__ of every vector kernel
-constexpr int kMaxDotBlocks = 4096;    // partial sums per Dot workspace slot
+constexpr int kMaxDotBlocks = 16384;   // partial sums per Dot workspace slot
 constexpr int kDotSlots = 32;          // Dot calls that may be in flight per device
 
 // Resolved launch shape for the register-vector kernels.
