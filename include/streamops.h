@@ -45,7 +45,8 @@ enum streamops_status {
     STREAMOPS_ERR_CUDA = 4,      /* a CUDA call failed; see streamops_last_cuda_error */
     STREAMOPS_ERR_WORKSPACE = 5, /* the per-device workspace could not be created */
     STREAMOPS_ERR_TIMEOUT = 6,   /* a bounded wait inside a bulk-copy kernel gave up */
-    STREAMOPS_ERR_ARG = 7        /* an argument outside its documented range */
+    STREAMOPS_ERR_ARG = 7,       /* an argument outside its documented range */
+    STREAMOPS_ERR_TOO_LARGE = 8  /* n exceeds what the fixed scratch of stream_dot_noalloc_f64 covers */
 };
 
 enum streamops_op { STREAMOPS_COPY = 0, STREAMOPS_SCALE = 1, STREAMOPS_ADD = 2,
@@ -83,6 +84,30 @@ int stream_triad_f32(const float *x, const float *y, float *out, double scalar, 
 int stream_dot_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
 int stream_dot_f32(const float *x, const float *y, float *out, double scalar, size_t n, streamops_stream_t stream);
 #define STREAMOPS_DOT_SLOTS 32
+
+/* Dot without any allocation (the paper has no counterpart; this entry point exists for callers
+ * that cannot allocate device memory when they need the result: code that runs after a memory
+ * pool has taken the whole device, loops that must not take the allocator's lock or trigger its
+ * implicit synchronisation, hosts whose rule is that libraries do not allocate).
+ * Same contract as stream_dot_f64 -- device pointers, asynchronous on `stream`, out[0] receives the
+ * fp64 dot product, same fixed-order summation so repeated calls give identical bits, same
+ * accuracy -- with these differences:
+ *   - The partial sums live in a fixed 33,024-byte array inside the library image instead of the
+ *     allocated workspace. Every GPU that loads the library holds that array until the process
+ *     exits. The call path runs no cudaMalloc, cudaFree or allocating library routine, and does
+ *     not create the workspace of streamops_init.
+ *   - n may not exceed STREAMOPS_DOT_NOALLOC_MAX_N (2^28 elements, 2 GiB per input): each partial
+ *     sum covers a fixed span of 65,536 elements and the array holds 4,096 of them. Larger n
+ *     returns STREAMOPS_ERR_TOO_LARGE and launches nothing.
+ *   - One array per device, shared by every call and every stream, keeping the previous call's
+ *     contents (the entry point re-zeroes the part that must start at zero). Two calls that
+ *     overlap in time on one GPU race on it and give wrong results: keep them on one stream or
+ *     order them with events.
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current). Make that first call outside stream capture.
+ * The summation order differs from stream_dot_f64's, so the two agree to rounding, not bitwise. */
+int stream_dot_noalloc_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
+#define STREAMOPS_DOT_NOALLOC_MAX_N (1ull << 28)
 
 /* One pass of the five kernels over three HOST arrays of n elements each, in the textbook
  * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The three arrays are

@@ -369,6 +369,7 @@ const char *streamops_status_string(int status) {
         case STREAMOPS_ERR_WORKSPACE: return "workspace allocation failed";
         case STREAMOPS_ERR_TIMEOUT: return "a bounded wait inside a kernel gave up";
         case STREAMOPS_ERR_ARG: return "argument out of range";
+        case STREAMOPS_ERR_TOO_LARGE: return "n exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

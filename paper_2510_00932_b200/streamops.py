@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
                 f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
             f = getattr(L, f"streamops_chain_host_{t}")
             f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
+        L.stream_dot_noalloc_f64.argtypes, L.stream_dot_noalloc_f64.restype = [vp, vp, vp, dbl, sz, vp], ci
         L.streamops_init.argtypes, L.streamops_init.restype = [ci], ci
         L.streamops_shutdown.argtypes, L.streamops_shutdown.restype = [], ci
         L.streamops_set_tuning.argtypes, L.streamops_set_tuning.restype = [ci, ci, ctypes.POINTER(Tuning)], ci
@@ -151,6 +152,24 @@ def dot(x, y, out, scalar: float = 0.0):
     if x.numel() != y.numel() or out.numel() != 1:
         raise ValueError("dot takes two equal-length inputs and a one-element output")
     _raise(getattr(lib(), f"stream_dot_{suf}")(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+DOT_NOALLOC_MAX_N = 1 << 28
+
+
+def dot_noalloc(x, y, out, scalar: float = 0.0):
+    """fp64 Dot through stream_dot_noalloc_f64: for callers that cannot allocate device memory
+    (the whole device already belongs to a pool, or the allocator's lock and implicit
+    synchronisation are off limits where the result is needed). The partial sums sit in a fixed
+    array inside the library, so n is limited to DOT_NOALLOC_MAX_N and calls that overlap in time
+    on one GPU race; make the first call on a device outside stream capture."""
+    suf, stream = _marshal(x, y, out)
+    if suf != "f64":
+        raise TypeError("the no-allocation Dot is fp64 only")
+    if x.numel() != y.numel() or out.numel() != 1:
+        raise ValueError("dot takes two equal-length inputs and a one-element output")
+    _raise(lib().stream_dot_noalloc_f64(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
     return out
 
 
