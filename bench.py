@@ -31,11 +31,12 @@ UNIT = "GB/s"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # an ncu capture, keyed by (workload, op, tuning signature); absent = not captured for this build.
 NCU_TRAFFIC_BYTES: dict = {
-    # profiles/ncu_full_five_kernels_c2_fp64.md: triad read 536.887 MB + write 229.862 MB (cold L2)
-    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "policy": 4, '
-                    '"stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 766_748_928,
-    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "policy": 4, '
-                  '"stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 769_038_080,
+    # profiles/ncu_chain_dram_c2_fp64.md (L2 state kept between kernels, as in the timed loop):
+    # add reads 477.2 MB + writes 270.2 MB; triad reads 477.4 MB + writes 268.1 MB per launch
+    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "pdl": 1, "policy": 5, '
+                  '"reverse": 0, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 747_400_000,
+    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "pdl": 1, "policy": 5, '
+                    '"reverse": 1, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 745_500_000,
 }
 
 
@@ -179,14 +180,26 @@ def run_ours(args):
             f()
     barrier()
 
-    # timed region: K steps, an event before every launch and one after the last
+    # timed region 1: K chain steps back to back, one event pair around all of them -> `value`
     sampler = harness.ClockSampler(gpu_index=local_rank).start() if rank == 0 else None
     time.sleep(0.3 if sampler else 0.0)
     K = args.steps
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(K)]
     launches0 = so.launch_count()
+    e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     first = sampler.mark() if sampler else 0
+    e_begin.record(stream)
+    for k in range(K):
+        for _, f in calls:
+            f()
+    e_end.record(stream)
+    barrier()
+    elapsed_ms = e_begin.elapsed_time(e_end)
+    launches = so.launch_count() - launches0             # kernels launched inside region 1
+
+    # timed region 2: K more chain steps with an event before every launch -> per-kernel durations
+    # in chain order (the extra events cost ~2 us per launch, which is why region 1 has none)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(K)]
     for k in range(K):
         for i, (_, f) in enumerate(calls):
             events[k][i].record(stream)
@@ -194,14 +207,12 @@ def run_ours(args):
         events[k][-1].record(stream)
     barrier()
     last = sampler.mark() if sampler else 0
-    launches = so.launch_count() - launches0
     so.check()
-    elapsed_ms = events[0][0].elapsed_time(events[-1][-1])
     op_ms = {name: statistics.fmean(events[k][i].elapsed_time(events[k][i + 1]) for k in range(K))
              for i, (name, _) in enumerate(calls)}
     op_ms_best = {name: min(events[k][i].elapsed_time(events[k][i + 1]) for k in range(K))
                   for i, (name, _) in enumerate(calls)}
-    # sustained clocks: keep sampling through a short extra burst if the region was too brief
+    # sustained clocks: keep sampling through a short extra burst if the regions were too brief
     if sampler and last - first < 3:
         t_end = time.perf_counter() + 0.6
         while time.perf_counter() < t_end:
@@ -216,7 +227,7 @@ def run_ours(args):
     value, max_ms = harness.whole_job_gbs(harness.step_bytes(n, itemsize) * K, elapsed_ms, device)
     ms_per_step = max_ms / K
 
-    # second timed region, op-major: each kernel K times back to back, so that every launch pays
+    # timed region 3, op-major: each kernel K times back to back, so that every launch pays
     # for its own write-backs and none inherits cached or dirty lines from a different kernel
     iso_ms = {}
     for name, f in calls:
@@ -230,7 +241,7 @@ def run_ours(args):
         e1.record(stream)
         torch.cuda.synchronize(device)
         iso_ms[name] = harness.max_over_ranks(e0.elapsed_time(e1) / K, device)
-    launches = so.launch_count() - launches0
+    launches_all = so.launch_count() - launches0
 
     # end to end: host buffers in, host buffers out, through the library's host entry point
     ha, hb, hc = (p.numpy() for p in pinned)
@@ -255,7 +266,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": per_op[dominant]["gbs"], "peak": peak,
                 "peak_source": f"of {peak_src}", "unit": "GB/s",
                 "frac": round(per_op[dominant]["gbs"] / peak, 4), "traffic": traffic,
-                "region": "chain-order steps; per_op_isolated has the same kernels timed op-major"}
+                "region": "chain-order steps with per-launch events; per_op_isolated = same kernels op-major"}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and args.cpu_seconds > 0:
@@ -275,7 +286,7 @@ def run_ours(args):
             "clocks": clocks, "per_op": per_op, "per_op_isolated": per_op_isolated, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": 3 * n * itemsize,
                     "d2h_bytes_per_step": 3 * n * itemsize + itemsize, "steps": e2e_steps},
-            "gpu_launches": int(launches), "frac_nominal_8tbs": round(value / world / harness.NOMINAL_HBM_GBS, 4),
+            "gpu_launches": int(launches), "gpu_launches_all_regions": int(launches_all), "frac_nominal_8tbs": round(value / world / harness.NOMINAL_HBM_GBS, 4),
             "tuning": sig,
         }
         print(json.dumps(line), flush=True)

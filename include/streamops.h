@@ -137,11 +137,16 @@ typedef struct streamops_tuning {
     int unroll;         /* kind 0: vectors per thread per array in flight: 1, 2 or 4 */
     int threads;        /* threads per block: 128, 256 or 512 (kind 1: consumer threads) */
     int blocks_per_sm;  /* persistent grid = blocks_per_sm * SMs; 0 = one block per tile */
-    int policy;         /* kind 0 cache-hint set, 0..4 (see streamops_policy_name) */
+    int policy;         /* kind 0 cache-hint set, 0..6 (see streamops_policy_name) */
     int contiguous;     /* 0 = tiles interleaved across blocks, 1 = one contiguous range per block */
     int chunk_bytes;    /* kind 1: bytes per bulk copy per array (multiple of 16, <= 65536) */
     int stages;         /* kind 1: ring depth, 2..8 */
     int two_pass;       /* Dot only: 1 = second pass as its own launch, 0 = last block finishes */
+    int reverse;        /* kind 0: 1 = walk the array from its end to its start (L2 reuse when the
+                           previous kernel wrote this kernel's input front to back) */
+    int pdl;            /* kind 0: 1 = programmatic dependent launch: the kernel's blocks may become
+                           resident while the previous kernel of the stream drains, and wait inside
+                           the kernel until it has completed (hides launch latency) */
 } streamops_tuning_t;
 
 int streamops_set_tuning(int op, int dtype, const streamops_tuning_t *t);

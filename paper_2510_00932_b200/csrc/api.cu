@@ -35,17 +35,24 @@ std::atomic<unsigned long long> g_launches{0};
 // Defaults: the measured best launch shapes on B200 for arrays far larger than L2 (fp64 n = 2^25,
 // fp32 n = 2^26). The elementwise kernels run one block per tile: the hardware block scheduler
 // then balances the two dies' unequal distance to memory better than a static persistent grid.
+// L2 use across consecutive kernels: loads are marked evict-first (read-once data) while stores
+// keep the normal priority (the next kernel usually reads what this one wrote), and scale and
+// triad walk their arrays from the end, so that in the sequence copy, scale, add, triad, dot every
+// kernel starts where its producer stopped and finds the producer's last ~55 MB still in L2
+// (measured: 14 % fewer DRAM reads per pass of the five kernels at fp64 n = 2^25). Programmatic
+// dependent launch is on: back-to-back kernels of one stream overlap launch latency with the
+// predecessor's tail (measured: 2 us per launch).
 streamops_tuning_t default_tuning(int op, int dtype) {
     streamops_tuning_t t;
     t.kind = 0; t.vec_bytes = 32; t.unroll = 2; t.threads = 256; t.blocks_per_sm = 0;
-    t.policy = 0; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0;
+    t.policy = 5; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0; t.reverse = 0; t.pdl = 1;
     const bool f64 = dtype == DT_F64;
     switch (op) {
         case OP_COPY:  t.unroll = 4; break;
-        case OP_SCALE: if (f64) { t.policy = 4; } else { t.unroll = 4; t.policy = 2; } break;
-        case OP_ADD:   t.threads = 128; if (f64) { t.policy = 4; } else { t.unroll = 4; } break;
-        case OP_TRIAD: t.threads = 128; t.policy = 4; break;
-        case OP_DOT:   t.threads = 512; t.blocks_per_sm = 2; if (f64) { t.unroll = 4; } else { t.unroll = 1; t.policy = 2; } break;
+        case OP_SCALE: t.reverse = 1; if (!f64) t.unroll = 4; break;
+        case OP_ADD:   t.threads = 128; if (!f64) t.unroll = 4; break;
+        case OP_TRIAD: t.threads = 128; t.reverse = 1; break;
+        case OP_DOT:   t.threads = 512; t.blocks_per_sm = 2; t.policy = 4; t.unroll = f64 ? 4 : 1; break;
     }
     return t;
 }
@@ -150,6 +157,8 @@ VecLaunch resolve_vec(const streamops_tuning_t &t, const DeviceState &d, int op,
     c.unroll = t.unroll;
     c.threads = t.threads;
     c.contiguous = t.contiguous;
+    c.reverse = t.reverse != 0;
+    c.pdl = t.pdl != 0;
     c.policy = t.policy;
     // the read-only data path must not be used on an array the kernel also writes
     if (c.policy == 1 && (out == x || out == y)) c.policy = 0;
@@ -168,7 +177,7 @@ bool valid_tuning(const streamops_tuning_t &t) {
     if (t.unroll != 1 && t.unroll != 2 && t.unroll != 4) return false;
     if (t.threads != 128 && t.threads != 256 && t.threads != 512) return false;
     if (t.blocks_per_sm < 0 || t.blocks_per_sm > 32) return false;
-    if (t.policy < 0 || t.policy > 4) return false;
+    if (t.policy < 0 || t.policy > 6) return false;
     if (t.chunk_bytes < 1024 || t.chunk_bytes > 65536 || (t.chunk_bytes & 15)) return false;
     if (t.stages < 2 || t.stages > 8) return false;
     return true;
@@ -342,6 +351,8 @@ const char *streamops_policy_name(int policy) {
         case 2: return "ld.global.cs / st.global.cs";
         case 3: return "ld.global.L1::no_allocate / st.global.cs";
         case 4: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first";
+        case 5: return "ld.global.L1::no_allocate + L2 evict_first / st.global";
+        case 6: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_last";
         default: return "unknown";
     }
 }

@@ -30,14 +30,14 @@ __device__ __forceinline__ double fold_vec(double acc, const Vec<VB> &xv, const 
 
 template <typename T, int VB, int U, int POL, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads)
-dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out) {
+dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int reverse) {
     constexpr int EPV = VB / (int)sizeof(T);
     __shared__ double warp_part[32];
     __shared__ bool is_last;
+    grid_dependency_sync();
     const char *xb = reinterpret_cast<const char *>(x);
     const char *yb = reinterpret_cast<const char *>(y);
-    uint64_t l2pol = 0;
-    if constexpr (POL == 4) l2pol = make_evict_first_policy();
+    const uint64_t l2pol = make_l2_policies<POL>().ld;
 
     const size_t nvec = n / EPV;
     const size_t tile_vecs = (size_t)blockDim.x * U;
@@ -47,7 +47,7 @@ dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *t
     for (int u = 0; u < U; ++u) acc[u] = 0.0;
 
     for (size_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const size_t v0 = tile * tile_vecs + threadIdx.x;
+        const size_t v0 = (reverse ? ntiles - 1 - tile : tile) * tile_vecs + threadIdx.x;
         Vec<VB> xv[U], yv[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
@@ -98,8 +98,8 @@ dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *
 template <typename T, int VB, int U, bool SL>
 cudaError_t launch_pol(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
     switch (c.policy) {
-#define STREAMOPS_CASE(P) case P: dot_pass1_kernel<T, VB, U, P, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out); break;
-        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4)
+#define STREAMOPS_CASE(P) case P: return launch_kernel(dot_pass1_kernel<T, VB, U, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, c.reverse);
+        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4) STREAMOPS_CASE(5) STREAMOPS_CASE(6)
 #undef STREAMOPS_CASE
         default: return cudaErrorInvalidValue;
     }

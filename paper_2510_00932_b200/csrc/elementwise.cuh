@@ -5,7 +5,9 @@
 // contiguous 512- or 1024-byte span. A thread issues all of a tile's loads (U per input array)
 // before the first arithmetic instruction: U * VB bytes per array per thread are in flight,
 // which is what hides HBM latency. Blocks walk the tiles either interleaved (tile b, b + G,
-// ...) or as one contiguous range per block. The ragged end -- vectors past the last full tile,
+// ...) or as one contiguous range per block, from the low addresses up or -- "reverse" -- from the
+// high addresses down (a kernel that consumes what the previous kernel just wrote finds the most
+// recently written lines still in L2 if it starts where the producer stopped). The ragged end -- vectors past the last full tile,
 // then elements past the last full vector -- is handled by one block with bounds checks, using
 // the same arithmetic.
 //
@@ -46,13 +48,13 @@ __device__ __forceinline__ void apply_vec(Vec<VB> &xv, const Vec<VB> &yv, T s) {
 
 template <typename T, int OP, int VB, int U, int POL>
 __global__ void __launch_bounds__(kMaxThreads)
-ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous) {
+ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int reverse) {
     constexpr int EPV = VB / (int)sizeof(T);
+    grid_dependency_sync();
     const char *xb = reinterpret_cast<const char *>(x);
     const char *yb = reinterpret_cast<const char *>(y);
     char *ob = reinterpret_cast<char *>(out);
-    uint64_t l2pol = 0;
-    if constexpr (POL == 4) l2pol = make_evict_first_policy();
+    const L2Policies l2 = make_l2_policies<POL>();
 
     const size_t nvec = n / EPV;
     const size_t tile_vecs = (size_t)blockDim.x * U;
@@ -67,18 +69,18 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous) {
         tile = blockIdx.x; end = ntiles; step = gridDim.x;
     }
     for (; tile < end; tile += step) {
-        const size_t v0 = tile * tile_vecs + threadIdx.x;
+        const size_t v0 = (reverse ? ntiles - 1 - tile : tile) * tile_vecs + threadIdx.x;
         Vec<VB> xv[U], yv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+        for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
         if constexpr (kUsesY<OP>) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+            for (int u = 0; u < U; ++u) ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             apply_vec<T, OP, VB>(xv[u], yv[u], s);
-            stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], l2pol);
+            stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], l2.st);
         }
     }
     // ragged end, by the block that is next in line for a tile
@@ -117,8 +119,8 @@ template <> struct WordOf<float> { using type = unsigned int; };
 template <typename T, int OP, int VB, int U>
 cudaError_t launch_vec_pol(const VecLaunch &c, const T *x, const T *y, T *out, T s, size_t n, cudaStream_t st) {
     switch (c.policy) {
-#define STREAMOPS_CASE(P) case P: ew_vec_kernel<T, OP, VB, U, P><<<c.grid, c.threads, 0, st>>>(x, y, out, s, n, c.contiguous); break;
-        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4)
+#define STREAMOPS_CASE(P) case P: return launch_kernel(ew_vec_kernel<T, OP, VB, U, P>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, out, s, n, c.contiguous, c.reverse);
+        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4) STREAMOPS_CASE(5) STREAMOPS_CASE(6)
 #undef STREAMOPS_CASE
         default: return cudaErrorInvalidValue;
     }

@@ -21,6 +21,8 @@ struct VecLaunch {
     int threads;
     unsigned grid;
     int contiguous;
+    int reverse;       // 1 = walk the tiles from the high addresses down
+    int pdl;           // 1 = launch with programmatic stream serialization
 };
 
 // Resolved launch shape for the bulk-copy (TMA) pipeline kernels.
@@ -30,6 +32,35 @@ struct BulkLaunch {
     int chunk_bytes;
     int stages;
 };
+
+// Launch helper. With `pdl` the kernel is launched with programmatic stream serialization: its
+// blocks may become resident while the previous kernel in the stream is still draining, and
+// wait at grid_dependency_wait() until that kernel has completed and its writes are visible.
+// That hides the launch latency and block-scheduling ramp between dependent kernels.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                 cudaStream_t stream, bool pdl, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+#ifdef __CUDACC__
+// First statements of every kernel that may be launched with `pdl`: let the next kernel in the
+// stream start launching, then wait for the previous one (both are no-ops in a plain launch).
+__device__ __forceinline__ void grid_dependency_sync() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
 
 // Per-slot Dot scratch: partial sums written by pass 1, the arrival ticket of the single-launch
 // variant, and (shared) the device error flag.

@@ -7,6 +7,8 @@
 //   2  ld.global.cs                 st.global.cs                   (evict-first streaming)
 //   3  ld.global.L1::no_allocate    st.global.cs
 //   4  ld.global.L1::no_allocate + L2 evict_first policy on loads and stores
+//   5  loads as 4 (read-once data leaves L2 first), plain st.global (written data stays)
+//   6  loads as 4, stores with an L2 evict_last policy (written data is kept for the next kernel)
 // 16-byte accesses are .v4.b32; 32-byte accesses are the 256-bit .v8.b32 form of sm_100.
 #pragma once
 #include <cstdint>
@@ -14,7 +16,7 @@
 
 namespace streamops {
 
-constexpr int kNumPolicies = 5;
+constexpr int kNumPolicies = 7;
 
 template <int VB> struct Vec;
 template <> struct alignas(16) Vec<16> { uint32_t w[4]; };
@@ -24,6 +26,20 @@ __device__ __forceinline__ uint64_t make_evict_first_policy() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     return pol;
+}
+__device__ __forceinline__ uint64_t make_evict_last_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// The L2 policy operands a kernel needs for its policy: one for loads, one for stores.
+struct L2Policies { uint64_t ld, st; };
+template <int POL> __device__ __forceinline__ L2Policies make_l2_policies() {
+    L2Policies p{0, 0};
+    if constexpr (POL >= 4) p.ld = make_evict_first_policy();
+    if constexpr (POL == 4) p.st = p.ld;
+    if constexpr (POL == 6) p.st = make_evict_last_policy();
+    return p;
 }
 
 #define STREAMOPS_LD16(QUAL, TAIL, ...)                                                          \
@@ -51,7 +67,7 @@ __device__ __forceinline__ void ldg(Vec<16> &v, const void *p, uint64_t l2pol) {
     else if constexpr (POL == 1) STREAMOPS_LD16(".nc", "");
     else if constexpr (POL == 2) STREAMOPS_LD16(".cs", "");
     else if constexpr (POL == 3) STREAMOPS_LD16(".L1::no_allocate", "");
-    else STREAMOPS_LD16(".L1::no_allocate.L2::cache_hint", ", %5", , "l"(l2pol));
+    else STREAMOPS_LD16(".L1::no_allocate.L2::cache_hint", ", %5", , "l"(l2pol));   // 4, 5, 6
 }
 template <int POL>
 __device__ __forceinline__ void ldg(Vec<32> &v, const void *p, uint64_t l2pol) {
@@ -63,13 +79,13 @@ __device__ __forceinline__ void ldg(Vec<32> &v, const void *p, uint64_t l2pol) {
 }
 template <int POL>
 __device__ __forceinline__ void stg(void *p, const Vec<16> &v, uint64_t l2pol) {
-    if constexpr (POL == 0 || POL == 1) STREAMOPS_ST16("", "");
+    if constexpr (POL == 0 || POL == 1 || POL == 5) STREAMOPS_ST16("", "");
     else if constexpr (POL == 2 || POL == 3) STREAMOPS_ST16(".cs", "");
     else STREAMOPS_ST16(".L2::cache_hint", ", %5", , "l"(l2pol));
 }
 template <int POL>
 __device__ __forceinline__ void stg(void *p, const Vec<32> &v, uint64_t l2pol) {
-    if constexpr (POL == 0 || POL == 1) STREAMOPS_ST32("", "");
+    if constexpr (POL == 0 || POL == 1 || POL == 5) STREAMOPS_ST32("", "");
     else if constexpr (POL == 2 || POL == 3) STREAMOPS_ST32(".cs", "");
     else STREAMOPS_ST32(".L2::cache_hint", ", %9", , "l"(l2pol));
 }
