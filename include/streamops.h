@@ -109,6 +109,16 @@ int stream_dot_f32(const float *x, const float *y, float *out, double scalar, si
 int stream_dot_noalloc_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
 #define STREAMOPS_DOT_NOALLOC_MAX_N (1ull << 28)
 
+/* One pass of the five kernels over three DEVICE arrays of n elements each, in the textbook
+ * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot_out[0] <- dot(a, b). Exactly the five
+ * stream_* calls above issued back to back on `stream` (asynchronous, nothing synchronised), from
+ * one library call: at L2-resident sizes -- the paper's ARRAY_SIZE values, Table 1 -- the host's
+ * per-call cost is what limits an iteration, and the edits the paper reports for these kernels
+ * (Table 2) were all on that side. The sequence can be captured into a CUDA graph (call
+ * streamops_init first: capture must not allocate). a, b, c must be distinct arrays. */
+int streamops_chain_f64(double *a, double *b, double *c, double *dot_out, double scalar, size_t n, streamops_stream_t stream);
+int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double scalar, size_t n, streamops_stream_t stream);
+
 /* One pass of the five kernels over three HOST arrays of n elements each, in the textbook
  * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The three arrays are
  * copied to the device, the five kernels above run on them, and the three arrays and the dot

@@ -292,6 +292,25 @@ STREAMOPS_BINARY(stream_triad_f32, OP_TRIAD, float, DT_F32)
 STREAMOPS_BINARY(stream_dot_f64, OP_DOT, double, DT_F64)
 STREAMOPS_BINARY(stream_dot_f32, OP_DOT, float, DT_F32)
 
+// Device-pointer chain: five asynchronous launches from one call.
+static int chain_device(int dtype, void *a, void *b, void *c, void *dot_out, double scalar, size_t n,
+                        streamops_stream_t stream) {
+    int status;
+    if ((status = run_op(OP_COPY, dtype, a, nullptr, c, scalar, n, stream)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_SCALE, dtype, c, nullptr, b, scalar, n, stream)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_ADD, dtype, a, b, c, scalar, n, stream)) != STREAMOPS_OK) return status;
+    if ((status = run_op(OP_TRIAD, dtype, b, c, a, scalar, n, stream)) != STREAMOPS_OK) return status;
+    return run_op(OP_DOT, dtype, a, b, dot_out, scalar, n, stream);
+}
+int streamops_chain_f64(double *a, double *b, double *c, double *dot_out, double scalar, size_t n,
+                        streamops_stream_t stream) {
+    return chain_device(DT_F64, a, b, c, dot_out, scalar, n, stream);
+}
+int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double scalar, size_t n,
+                        streamops_stream_t stream) {
+    return chain_device(DT_F32, a, b, c, dot_out, scalar, n, stream);
+}
+
 int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out) {
     return chain_host<double>(a, b, c, scalar, n, dot_out);
 }

@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
                 f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
             f = getattr(L, f"streamops_chain_host_{t}")
             f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
+            f = getattr(L, f"streamops_chain_{t}")
+            f.argtypes, f.restype = [vp, vp, vp, vp, dbl, sz, vp], ci
         L.stream_dot_noalloc_f64.argtypes, L.stream_dot_noalloc_f64.restype = [vp, vp, vp, dbl, sz, vp], ci
         L.streamops_init.argtypes, L.streamops_init.restype = [ci], ci
         L.streamops_shutdown.argtypes, L.streamops_shutdown.restype = [], ci
@@ -85,29 +87,40 @@ def _raise(status: int):
         raise StreamopsError(status, msg)
 
 
+_SUFFIX = None            # torch dtype -> "f32" / "f64", filled on first use
+_raw_stream = None        # fast accessor of the current stream's handle
+
+
 def _suffix(t) -> str:
-    import torch
-    if t.dtype == torch.float64:
-        return "f64"
-    if t.dtype == torch.float32:
-        return "f32"
-    raise TypeError(f"libstreamops handles float32 and float64 tensors, got {t.dtype}")
+    global _SUFFIX
+    if _SUFFIX is None:
+        import torch
+        _SUFFIX = {torch.float64: "f64", torch.float32: "f32"}
+    try:
+        return _SUFFIX[t.dtype]
+    except KeyError:
+        raise TypeError(f"libstreamops handles float32 and float64 tensors, got {t.dtype}") from None
 
 
 def _marshal(*tensors):
-    """Common dtype suffix, element count and the current stream of the tensors' device."""
-    import torch
+    """Common dtype suffix and the current stream handle of the tensors' device. Kept lean: at
+    L2-resident sizes a kernel lasts a few microseconds and this code is what the host spends."""
+    global _raw_stream
     first = tensors[0]
     suf = _suffix(first)
+    dev = first.get_device()
     for t in tensors:
         if not t.is_cuda:
             raise ValueError("libstreamops operates on CUDA tensors")
-        if not t.is_contiguous() or t.dim() != 1:
+        if t.dim() != 1 or not t.is_contiguous():
             raise ValueError("libstreamops operates on contiguous 1-D tensors")
-        if _suffix(t) != suf or t.device != first.device:
+        if t.dtype != first.dtype or t.get_device() != dev:
             raise ValueError("all tensors of one call share dtype and device")
-    stream = torch.cuda.current_stream(first.device).cuda_stream
-    return suf, stream
+    if _raw_stream is None:
+        import torch
+        _raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None) or (
+            lambda d: torch.cuda.current_stream(d).cuda_stream)
+    return suf, _raw_stream(dev)
 
 
 def copy(x, out, scalar: float = 0.0):
@@ -175,12 +188,13 @@ def dot_noalloc(x, y, out, scalar: float = 0.0):
 
 def chain(a, b, c, dot_out, scalar: float):
     """One pass of the five kernels over device tensors a, b, c in the STREAM dataflow:
-    c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot_out <- dot(a, b). Five library calls."""
-    copy(a, c)
-    scale(c, b, scalar)
-    add(a, b, c)
-    triad(b, c, a, scalar)
-    dot(a, b, dot_out)
+    c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot_out <- dot(a, b) (streamops_chain_*: one library
+    call, five asynchronous launches)."""
+    suf, stream = _marshal(a, b, c, dot_out)
+    if not (a.numel() == b.numel() == c.numel()) or dot_out.numel() != 1:
+        raise ValueError("chain takes three equal-length arrays and a one-element output")
+    _raise(getattr(lib(), f"streamops_chain_{suf}")(a.data_ptr(), b.data_ptr(), c.data_ptr(), dot_out.data_ptr(),
+                                                   float(scalar), a.numel(), stream))
 
 
 def chain_host(a, b, c, scalar: float):
