@@ -32,11 +32,11 @@ UNIT = "GB/s"
 # an ncu capture, keyed by (workload, op, tuning signature); absent = not captured for this build.
 NCU_TRAFFIC_BYTES: dict = {
     # profiles/ncu_chain_dram_c2_fp64.md (L2 state kept between kernels, as in the timed loop):
-    # add reads 477.2 MB + writes 270.2 MB; triad reads 477.4 MB + writes 268.1 MB per launch
-    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "pdl": 1, "policy": 5, '
-                  '"reverse": 0, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 747_400_000,
-    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "kind": 0, "pdl": 1, "policy": 5, '
-                    '"reverse": 1, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 745_500_000,
+    # add reads 465.8 MB + writes 272.8 MB; triad reads 464.1 MB + writes 266.5 MB per launch
+    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "keep_mib": 112, "kind": 0, "pdl": 1, '
+                  '"policy": 7, "reverse": 0, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 738_600_000,
+    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "keep_mib": 112, "kind": 0, "pdl": 1, '
+                    '"policy": 7, "reverse": 1, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 730_600_000,
 }
 
 
@@ -48,6 +48,9 @@ def parse_args():
     p.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4"])
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--e2e-steps", type=int, default=5)
+    p.add_argument("--tuning", default="",
+                   help='JSON overrides of the launch tuning for A/B runs, e.g. \'{"ew": {"policy": 5}, "dot": {"two_pass": 1}}\' '
+                        '("ew" = copy, scale, add, triad; "all" = the five ops)')
     p.add_argument("--cpu-seconds", type=float, default=12.0,
                    help="CPU time budget of the oracle baseline leg (0 = skip)")
     return p.parse_args()
@@ -158,6 +161,9 @@ def run_ours(args):
     so.init(local_rank)
 
     w = inputs.WORKLOADS[args.workload]
+    for key, fields in (json.loads(args.tuning) if args.tuning else {}).items():
+        for op in {"ew": so.OPS[:4], "all": so.OPS}.get(key, (key,)):
+            so.set_tuning(op, w.dtype, **fields)
     # every rank works on its own replica of the workload (same recipe, rank-specific seed)
     wr = inputs.Workload(w.name, w.dtype, w.n, w.dist, w.seed + 1000 * rank, w.scalar, w.iterations)
     a, b, c = inputs.make_arrays(wr)

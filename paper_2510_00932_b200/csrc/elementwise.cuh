@@ -48,7 +48,7 @@ __device__ __forceinline__ void apply_vec(Vec<VB> &xv, const Vec<VB> &yv, T s) {
 
 template <typename T, int OP, int VB, int U, int POL>
 __global__ void __launch_bounds__(kMaxThreads)
-ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int reverse) {
+ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int reverse, size_t hot_tiles) {
     constexpr int EPV = VB / (int)sizeof(T);
     grid_dependency_sync();
     const char *xb = reinterpret_cast<const char *>(x);
@@ -70,6 +70,8 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int
     }
     for (; tile < end; tile += step) {
         const size_t v0 = (reverse ? ntiles - 1 - tile : tile) * tile_vecs + threadIdx.x;
+        // two-phase stores: the first hot_tiles tiles of the traversal leave L2 first
+        const uint64_t stpol = (POL >= 7 && tile >= hot_tiles) ? l2.st_late : l2.st;
         Vec<VB> xv[U], yv[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
@@ -80,7 +82,7 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             apply_vec<T, OP, VB>(xv[u], yv[u], s);
-            stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], l2.st);
+            stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], stpol);
         }
     }
     // ragged end, by the block that is next in line for a tile
@@ -119,8 +121,8 @@ template <> struct WordOf<float> { using type = unsigned int; };
 template <typename T, int OP, int VB, int U>
 cudaError_t launch_vec_pol(const VecLaunch &c, const T *x, const T *y, T *out, T s, size_t n, cudaStream_t st) {
     switch (c.policy) {
-#define STREAMOPS_CASE(P) case P: return launch_kernel(ew_vec_kernel<T, OP, VB, U, P>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, out, s, n, c.contiguous, c.reverse);
-        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4) STREAMOPS_CASE(5) STREAMOPS_CASE(6)
+#define STREAMOPS_CASE(P) case P: return launch_kernel(ew_vec_kernel<T, OP, VB, U, P>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, out, s, n, c.contiguous, c.reverse, c.hot_tiles);
+        STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4) STREAMOPS_CASE(5) STREAMOPS_CASE(6) STREAMOPS_CASE(7) STREAMOPS_CASE(8)
 #undef STREAMOPS_CASE
         default: return cudaErrorInvalidValue;
     }

@@ -23,6 +23,7 @@ struct VecLaunch {
     int contiguous;
     int reverse;       // 1 = walk the tiles from the high addresses down
     int pdl;           // 1 = launch with programmatic stream serialization
+    size_t hot_tiles;  // policies 7, 8: tiles at the start of the traversal whose stores are evict-first
 };
 
 // Resolved launch shape for the bulk-copy (TMA) pipeline kernels.

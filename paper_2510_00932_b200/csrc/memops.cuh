@@ -9,6 +9,11 @@
 //   4  ld.global.L1::no_allocate + L2 evict_first policy on loads and stores
 //   5  loads as 4 (read-once data leaves L2 first), plain st.global (written data stays)
 //   6  loads as 4, stores with an L2 evict_last policy (written data is kept for the next kernel)
+//   7  loads as 4; stores in two phases: L2 evict_first while the kernel is still consuming what
+//      its predecessor left in L2 (its own output must not push those lines out), normal
+//      priority afterwards (so that the kernel's last-written lines are what it leaves behind)
+//   8  as 7 with L2 evict_last in the second phase (the consumer's evict_first loads demote the
+//      lines again once they have been read)
 // 16-byte accesses are .v4.b32; 32-byte accesses are the 256-bit .v8.b32 form of sm_100.
 #pragma once
 #include <cstdint>
@@ -16,7 +21,7 @@
 
 namespace streamops {
 
-constexpr int kNumPolicies = 7;
+constexpr int kNumPolicies = 9;
 
 template <int VB> struct Vec;
 template <> struct alignas(16) Vec<16> { uint32_t w[4]; };
@@ -27,18 +32,26 @@ __device__ __forceinline__ uint64_t make_evict_first_policy() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
+__device__ __forceinline__ uint64_t make_evict_normal_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
 __device__ __forceinline__ uint64_t make_evict_last_policy() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
-// The L2 policy operands a kernel needs for its policy: one for loads, one for stores.
-struct L2Policies { uint64_t ld, st; };
+// The L2 policy operands a kernel needs for its policy: one for loads, one for stores, and for
+// the two-phase policy the one its stores switch to after the first phase.
+struct L2Policies { uint64_t ld, st, st_late; };
 template <int POL> __device__ __forceinline__ L2Policies make_l2_policies() {
-    L2Policies p{0, 0};
+    L2Policies p{0, 0, 0};
     if constexpr (POL >= 4) p.ld = make_evict_first_policy();
-    if constexpr (POL == 4) p.st = p.ld;
+    if constexpr (POL == 4 || POL == 7 || POL == 8) p.st = p.ld;
     if constexpr (POL == 6) p.st = make_evict_last_policy();
+    if constexpr (POL == 7) p.st_late = make_evict_normal_policy();
+    if constexpr (POL == 8) p.st_late = make_evict_last_policy();
     return p;
 }
 

@@ -44,7 +44,7 @@ def test_tuning_table_validation_needs_no_gpu(so):
     so.set_tuning("triad", "f64", unroll=4, policy=3)
     assert so.get_tuning("triad", "f64").unroll == 4
     assert so.get_tuning("triad", "f32").unroll == t.unroll          # per (op, dtype)
-    for bad in (dict(unroll=3), dict(vec_bytes=8), dict(threads=1024), dict(policy=7),
+    for bad in (dict(unroll=3), dict(vec_bytes=8), dict(threads=1024), dict(policy=9), dict(keep_mib=-1),
                 dict(stages=1), dict(chunk_bytes=1000), dict(kind=2)):
         with pytest.raises(so.StreamopsError) as e:
             so.set_tuning("triad", "f64", **bad)
