@@ -1,4 +1,5 @@
-"""CPU oracle for the five streaming kernels -- TEST INFRASTRUCTURE, not part of the product.
+"""CPU oracle for the five streaming kernels and the shared-memory exchange microkernel -- TEST
+INFRASTRUCTURE, not part of the product.
 
 Only ``tests/``, the smoke check and the benchmark's CPU-baseline leg may import this package.
 It wraps ``streamops_oracle.c`` (plain scalar C loops following the textbook definitions of the
@@ -16,7 +17,7 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = ["streamops_oracle.c", "streamops_oracle_mt.c"]
+_SOURCES = ["streamops_oracle.c", "streamops_oracle_mt.c", "shmem_oracle.c"]
 _LIB_PATH = os.path.join(_HERE, "liboracle.so")
 # contraction off: a*b+c must stay two rounded operations; no value-changing optimisation
 CFLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-pthread"]
@@ -60,6 +61,10 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_run_mt.argtypes = [ctypes.c_int, ctypes.c_int, dp, dp, dp, dbl, sz,
                                        ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
         _lib.oracle_run_mt.restype = ctypes.c_int
+        _lib.oracle_shmem_mix_u32.argtypes = [dp, dp, ctypes.c_uint, sz]
+        _lib.oracle_shmem_mix_u32.restype = None
+        _lib.oracle_shmem_mix_u32_mt.argtypes = [dp, dp, ctypes.c_uint, sz, ctypes.c_int]
+        _lib.oracle_shmem_mix_u32_mt.restype = ctypes.c_int
     return _lib
 
 
@@ -163,3 +168,24 @@ def chain(a: np.ndarray, b: np.ndarray, c: np.ndarray, scalar: float):
     c = add(a, b)
     a = triad(b, c, scalar)
     return a, b, c, dot(a, b)
+
+
+SHMEM_ROWS, SHMEM_COLS = 8, 1024
+SHMEM_TILE = SHMEM_ROWS * SHMEM_COLS
+
+
+def shmem_mix(x: np.ndarray, rounds: int, nthreads: int = 1) -> np.ndarray:
+    """Shared-memory exchange microkernel (the definition is in shmem_oracle.c): tiles of 8 rows
+    x 1024 columns of 32-bit words; a round adds to every row the row below it (cyclically, modulo
+    2^32); words past the last whole tile double every round. ``nthreads`` > 1 only deals whole
+    tiles to threads."""
+    if not (isinstance(x, np.ndarray) and x.dtype == np.uint32 and x.ndim == 1 and x.flags.c_contiguous):
+        raise ValueError("shmem_mix takes a contiguous 1-D uint32 array")
+    if rounds < 0 or rounds >= 2 ** 32:
+        raise ValueError("rounds out of range")
+    out = np.empty_like(x)
+    if nthreads <= 1:
+        lib().oracle_shmem_mix_u32(_p(x), _p(out), int(rounds), x.size)
+    elif lib().oracle_shmem_mix_u32_mt(_p(x), _p(out), int(rounds), x.size, int(nthreads)) != 0:
+        raise RuntimeError("oracle_shmem_mix_u32_mt failed")
+    return out

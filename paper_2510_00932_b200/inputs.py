@@ -111,3 +111,9 @@ def special_values(dtype: str) -> np.ndarray:
         0x3ECCCCCD, 0x4B000001,
     ], dtype=np.uint32)
     return bits.view(np.float32)
+
+
+def make_words(n: int, seed: int = 5) -> np.ndarray:
+    """Uniform random 32-bit words for the shared-memory exchange microkernel (PCG64 stream)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    return rng.integers(0, 1 << 32, size=int(n), dtype=np.uint32)
