@@ -51,6 +51,7 @@ def parse_args():
     p.add_argument("--tuning", default="",
                    help='JSON overrides of the launch tuning for A/B runs, e.g. \'{"ew": {"policy": 5}, "dot": {"two_pass": 1}}\' '
                         '("ew" = copy, scale, add, triad; "all" = the five ops)')
+    p.add_argument("--no-shmem", action="store_true", help="skip the shared-memory microkernel line")
     p.add_argument("--cpu-seconds", type=float, default=12.0,
                    help="CPU time budget of the oracle baseline leg (0 = skip)")
     return p.parse_args()
@@ -275,6 +276,28 @@ def run_ours(args):
     e2e_ms = (time.perf_counter() - t0) * 1e3
     e2e_value, _ = harness.whole_job_gbs(harness.step_bytes(n, itemsize) * e2e_steps, e2e_ms, device)
 
+    # the shared-memory exchange microkernel, at the paper's default repetition count (own line, not part of `value`)
+    shmem = None
+    if rank == 0 and world == 1 and not args.no_shmem:
+        from paper_2510_00932_b200 import shmembench
+        s2 = harness.ClockSampler(gpu_index=local_rank).start()
+        shmem = shmembench.measure(1 << 26, 600, 16, iters=20, device=device)
+        c2 = s2.summary(); s2.stop()
+        mhz = c2["sm_mhz"] or c2["sm_max_mhz"] or 1965.0
+        sms = torch.cuda.get_device_properties(device).multi_processor_count
+        shmem.update({"bound": "shared memory", "peak_gbs": round(shmembench.smem_peak_gbs(sms, mhz), 1),
+                      "peak_source": f"derived: 128 B/clk/SM x {sms} SMs x {mhz:.0f} MHz sampled during the launches",
+                      "frac": round(shmem["smem_gbs"] / shmembench.smem_peak_gbs(sms, mhz), 4), "sm_mhz": mhz})
+        if args.cpu_seconds > 0:
+            import oracle
+            nthreads = len(os.sched_getaffinity(0))
+            words = inputs.make_words(1 << 22)
+            oracle.shmem_mix(words, 8, nthreads)
+            t0 = time.perf_counter(); oracle.shmem_mix(words, 600, nthreads); dt = time.perf_counter() - t0
+            shmem["cpu_baseline"] = {"value": round(shmembench.smem_bytes(words.size, 600) / dt / 1e9, 2), "unit": "GB/s",
+                                     "cores": nthreads, "kind": "oracle",
+                                     "sample": "one all-threads pass over n=2^22 words, 600 rounds, same byte accounting"}
+
     peak, peak_src = harness.measured_peak()
     per_op = harness.per_op_report(op_ms, n, itemsize, peak)
     for name in per_op:
@@ -303,7 +326,7 @@ def run_ours(args):
             "config": {"workload": w.name, "n": n, "dist": w.dist, "seed": w.seed, "scalar": w.scalar,
                        "arrays": 3, "array_bytes": n * itemsize, "order": "chain (copy, scale, add, triad, dot per step)",
                        "l2": "no flush: each array is larger than the 126 MB L2", "parallelism": f"replicas x{world}"},
-            "clocks": clocks, "per_op": per_op, "per_op_isolated": per_op_isolated, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "clocks": clocks, "shmem_mix": shmem, "per_op": per_op, "per_op_isolated": per_op_isolated, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "e2e": {"value": round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": 3 * n * itemsize,
                     "d2h_bytes_per_step": 3 * n * itemsize + itemsize, "steps": e2e_steps},
             "gpu_launches": int(launches), "gpu_launches_all_regions": int(launches_all), "frac_nominal_8tbs": round(value / world / harness.NOMINAL_HBM_GBS, 4),

@@ -130,6 +130,25 @@ int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double sca
 int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out);
 int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out);
 
+/* Shared-memory exchange microkernel. Table 1 of the paper lists a shared-memory benchmark whose one
+ * parameter is a repetition count (300..1500, default 600) and whose time goes into shared-memory
+ * loads and stores (Table 2); the paper does not define it, so the operation is this library's own:
+ *   the n 32-bit words of x are cut into tiles of 8 rows x 1024 columns (row-major, 8192 words);
+ *   one round replaces, in every tile, row k by row k + row ((k + 1) mod 8), all eight rows taken
+ *   from the values before the round, addition modulo 2^32; a word past the last whole tile is a
+ *   row of its own and is doubled by a round; out = the array after `rounds` rounds.
+ * (Equivalently row k of the result is sum_j C(rounds, j) * row (k + j) mod 8.) Every round moves
+ * each word through shared memory once in each direction: 8 * rounds bytes of shared-memory
+ * traffic per word against 8 bytes of global traffic, so for rounds >> 5 the kernel is bound by
+ * shared-memory bandwidth (128 bytes per clock per SM).
+ * x and out are DEVICE pointers to n words, 4-byte aligned (16-byte alignment of both selects the
+ * widest shared-memory accesses), out == x allowed, any other overlap is STREAMOPS_ERR_OVERLAP;
+ * asynchronous on `stream`; n == 0 does nothing. streamops_set_shmem_width picks the width of one
+ * shared-memory access for A/B runs: 4, 8 or 16 bytes (default 16); the result does not depend on it. */
+int shmem_mix_u32(const unsigned *x, unsigned *out, unsigned rounds, size_t n, streamops_stream_t stream);
+int streamops_set_shmem_width(int bytes);
+int streamops_get_shmem_width(void);
+
 /* Creates the per-device state for `device` (SM count, the Dot workspace: partial sums, arrival
  * tickets, an error flag; a few MiB). Optional: every entry point does it on first use for the
  * current device. Allocates device memory, so call it outside stream capture. */

@@ -278,6 +278,11 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
 
 }  // namespace
 
+namespace streamops {
+int note_cuda_error(cudaError_t e) { return cuda_fail(e); }
+void note_launches(int n) { g_launches.fetch_add((unsigned long long)n); }
+}  // namespace streamops
+
 extern "C" {
 
 #define STREAMOPS_UNARY(NAME, OP, T, DT)                                                             \

@@ -70,6 +70,10 @@ struct DotScratch {
     unsigned *ticket;      // one counter, zero between calls
 };
 
+// api.cu: bookkeeping shared by the entry points that live in other files
+int note_cuda_error(cudaError_t e);      // records e, returns STREAMOPS_ERR_CUDA
+void note_launches(int n);              // adds to streamops_launch_count
+
 // elementwise.cu
 cudaError_t launch_elementwise(int op, int dtype, const VecLaunch &cfg, const void *x, const void *y,
                                void *out, double scalar, size_t n, cudaStream_t stream);

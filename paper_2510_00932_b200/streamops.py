@@ -61,6 +61,9 @@ def lib() -> ctypes.CDLL:
             f = getattr(L, f"streamops_chain_{t}")
             f.argtypes, f.restype = [vp, vp, vp, vp, dbl, sz, vp], ci
         L.stream_dot_noalloc_f64.argtypes, L.stream_dot_noalloc_f64.restype = [vp, vp, vp, dbl, sz, vp], ci
+        L.shmem_mix_u32.argtypes, L.shmem_mix_u32.restype = [vp, vp, ctypes.c_uint, sz, vp], ci
+        L.streamops_set_shmem_width.argtypes, L.streamops_set_shmem_width.restype = [ci], ci
+        L.streamops_get_shmem_width.argtypes, L.streamops_get_shmem_width.restype = [], ci
         L.streamops_init.argtypes, L.streamops_init.restype = [ci], ci
         L.streamops_shutdown.argtypes, L.streamops_shutdown.restype = [], ci
         L.streamops_set_tuning.argtypes, L.streamops_set_tuning.restype = [ci, ci, ctypes.POINTER(Tuning)], ci
@@ -184,6 +187,26 @@ def dot_noalloc(x, y, out, scalar: float = 0.0):
         raise ValueError("dot takes two equal-length inputs and a one-element output")
     _raise(lib().stream_dot_noalloc_f64(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
     return out
+
+
+def shmem_mix(x, out, rounds: int):
+    """out = x after `rounds` rounds of the shared-memory exchange (shmem_mix_u32): int32/uint32
+    CUDA tensors of equal length, treated as raw 32-bit words."""
+    import torch
+    for t in (x, out):
+        if not t.is_cuda or t.dim() != 1 or not t.is_contiguous() or t.element_size() != 4 or t.is_floating_point():
+            raise ValueError("shmem_mix operates on contiguous 1-D CUDA tensors of 32-bit integers")
+    if x.numel() != out.numel() or x.get_device() != out.get_device():
+        raise ValueError("length or device mismatch")
+    if not 0 <= int(rounds) < 2 ** 32:
+        raise ValueError("rounds out of range")
+    stream = torch.cuda.current_stream(x.get_device()).cuda_stream
+    _raise(lib().shmem_mix_u32(x.data_ptr(), out.data_ptr(), int(rounds), x.numel(), stream))
+    return out
+
+
+def set_shmem_width(width_bytes: int):
+    _raise(lib().streamops_set_shmem_width(int(width_bytes)))
 
 
 def chain(a, b, c, dot_out, scalar: float):

@@ -19,12 +19,12 @@ def so():
 def _declared_symbols():
     text = open(os.path.join(ROOT, "include", "streamops.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(stream_[a-z0-9_]+|streamops_[a-z0-9_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(stream_[a-z0-9_]+|streamops_[a-z0-9_]+|shmem_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_header_symbols_are_exported(so):
     names = _declared_symbols()
-    assert len(names) >= 22 and "stream_triad_f64" in names and "streamops_chain_host_f32" in names
+    assert len(names) >= 25 and "shmem_mix_u32" in names and "stream_triad_f64" in names and "streamops_chain_host_f32" in names
     L = so.lib()
     for n in names:
         assert hasattr(L, n), f"{n} declared in include/streamops.h but not exported"
