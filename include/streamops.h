@@ -85,6 +85,18 @@ int stream_dot_f64(const double *x, const double *y, double *out, double scalar,
 int stream_dot_f32(const float *x, const float *y, float *out, double scalar, size_t n, streamops_stream_t stream);
 #define STREAMOPS_DOT_SLOTS 32
 
+/* The two pieces a Dot over an array that is split across GPUs is made of (the sum is the only step
+ * of the five kernels that needs an exchange: one double per GPU).
+ * stream_dot_wide_f32: Dot of float arrays whose DEVICE output is the double-precision total before
+ * its final rounding to float, so that per-GPU partial results lose nothing (for double arrays
+ * stream_dot_f64 already is that). Always runs its second pass as a second launch.
+ * stream_fold_{f64,f32}: out[0] = (T)(((p[0] + p[1]) + p[2]) + ... + p[count-1]), the doubles added
+ * strictly left to right by one thread and rounded once to T: every GPU that folds the same
+ * gathered partial sums in rank order gets identical bits. count <= 2^24; count == 0 writes +0. */
+int stream_dot_wide_f32(const float *x, const float *y, double *out, double scalar, size_t n, streamops_stream_t stream);
+int stream_fold_f64(const double *partials, double *out, double scalar, size_t count, streamops_stream_t stream);
+int stream_fold_f32(const double *partials, float *out, double scalar, size_t count, streamops_stream_t stream);
+
 /* Dot without any allocation (the paper has no counterpart; this entry point exists for callers
  * that cannot allocate device memory when they need the result: code that runs after a memory
  * pool has taken the whole device, loops that must not take the allocator's lock or trigger its

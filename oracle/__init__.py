@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
                 getattr(_lib, f"oracle_{name}_{t}").restype = None
         _lib.oracle_dot_f64_longdouble.argtypes = [dp, dp, sz]
         _lib.oracle_dot_f64_longdouble.restype = dbl
+        _lib.oracle_fold_f64.argtypes = [dp, sz]
+        _lib.oracle_fold_f64.restype = dbl
         _lib.oracle_run_mt.argtypes = [ctypes.c_int, ctypes.c_int, dp, dp, dp, dbl, sz,
                                        ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
         _lib.oracle_run_mt.restype = ctypes.c_int
@@ -140,6 +142,14 @@ def dot_abs(x: np.ndarray, y: np.ndarray) -> float:
     """Sum of |x[i]*y[i]| (condition-number numerator)."""
     t = _check(x, y)
     return float(getattr(lib(), f"oracle_dot_abs_{t}")(_p(x), _p(y), x.size))
+
+
+def fold(partials: np.ndarray) -> float:
+    """Left-to-right double-precision sum of per-GPU partial dot products (rank order)."""
+    if not (isinstance(partials, np.ndarray) and partials.dtype == np.float64 and partials.ndim == 1
+            and partials.flags.c_contiguous):
+        raise ValueError("fold takes a contiguous 1-D float64 array")
+    return float(lib().oracle_fold_f64(_p(partials), partials.size))
 
 
 def run_mt(op: str, x: np.ndarray, y, scalar: float, nthreads: int, out=None):

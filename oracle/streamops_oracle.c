@@ -211,3 +211,14 @@ double oracle_dot_abs_f32(const float *x, const float *y, size_t n)
         acc += fabsl((long double)x[i] * (long double)y[i]);
     return (double)acc;
 }
+
+/* Fold of per-GPU partial sums (the exchange step of a Dot over an array split across GPUs):
+ * the doubles added strictly left to right, one rounding per addition; the caller rounds the
+ * total to the element type. */
+double oracle_fold_f64(const double *p, size_t count)
+{
+    double acc = 0.0;
+    for (size_t i = 0; i < count; ++i)
+        acc = acc + p[i];
+    return acc;
+}

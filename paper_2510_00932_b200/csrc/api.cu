@@ -124,16 +124,16 @@ bool ranges_overlap(const void *a, size_t abytes, const void *b, size_t bbytes) 
 }
 
 // Null / alignment / overlap rules common to the five operations.
-int check_args(int op, size_t esize, const void *x, const void *y, const void *out, size_t n) {
+int check_args(int op, size_t esize, const void *x, const void *y, const void *out, size_t n, size_t out_esize) {
     const bool uses_y = (op == OP_ADD || op == OP_TRIAD || op == OP_DOT);
     if (!out && (n > 0 || op == OP_DOT)) return STREAMOPS_ERR_NULL;   // Dot writes even for n == 0
     if (n > 0 && (!x || (uses_y && !y))) return STREAMOPS_ERR_NULL;
-    if (((uintptr_t)out % esize) || (n > 0 && (((uintptr_t)x % esize) || (uses_y && ((uintptr_t)y % esize)))))
+    if (((uintptr_t)out % out_esize) || (n > 0 && (((uintptr_t)x % esize) || (uses_y && ((uintptr_t)y % esize)))))
         return STREAMOPS_ERR_ALIGN;
     if (n == 0) return STREAMOPS_OK;
     if (n > ((size_t)1 << 48)) return STREAMOPS_ERR_ARG;
     const size_t bytes = n * esize;
-    const size_t obytes = (op == OP_DOT) ? esize : bytes;
+    const size_t obytes = (op == OP_DOT) ? out_esize : bytes;
     const void *ins[2] = {x, uses_y ? y : nullptr};
     for (const void *in : ins) {
         if (!in) continue;
@@ -189,15 +189,17 @@ bool valid_tuning(const streamops_tuning_t &t) {
     return true;
 }
 
+// `wide` (Dot only): out is one double receiving the unrounded total.
 int run_op(int op, int dtype, const void *x, const void *y, void *out, double scalar, size_t n,
-           streamops_stream_t stream_) {
+           streamops_stream_t stream_, bool wide = false) {
     cudaStream_t stream = (cudaStream_t)stream_;
     const size_t esize = dtype == DT_F64 ? 8 : 4;
-    int status = check_args(op, esize, x, y, out, n);
+    const size_t out_esize = wide ? 8 : esize;
+    int status = check_args(op, esize, x, y, out, n, out_esize);
     if (status != STREAMOPS_OK) return status;
     if (n == 0) {
         if (op != OP_DOT) return STREAMOPS_OK;
-        cudaError_t e = cudaMemsetAsync(out, 0, esize, stream);   // +0 in either format
+        cudaError_t e = cudaMemsetAsync(out, 0, out_esize, stream);   // +0 in either format
         return e == cudaSuccess ? STREAMOPS_OK : cuda_fail(e);
     }
     DeviceState *d = nullptr;
@@ -216,7 +218,7 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
     const bool uses_y = (op == OP_ADD || op == OP_TRIAD || op == OP_DOT);
     uintptr_t bits = (uintptr_t)x | (op == OP_DOT ? 0 : (uintptr_t)out);
     if (uses_y) bits |= (uintptr_t)y;
-    if (t.kind == 1 && !(bits & 15)) {
+    if (t.kind == 1 && !(bits & 15) && !wide) {
         BulkLaunch b;
         b.threads = t.threads;
         b.chunk_bytes = t.chunk_bytes;
@@ -229,7 +231,7 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
         e = launch_bulk(op, dtype, b, x, y, out, scalar, n, scratch, d->error_flag, stream, &launches);
     } else {
         const VecLaunch c = resolve_vec(t, *d, op, esize, x, y, out, n);
-        if (op == OP_DOT) e = launch_dot(dtype, c, t.two_pass != 0, x, y, out, n, scratch, stream, &launches);
+        if (op == OP_DOT) e = launch_dot(dtype, c, t.two_pass != 0, wide, x, y, out, n, scratch, stream, &launches);
         else e = launch_elementwise(op, dtype, c, x, y, out, scalar, n, stream);
     }
     if (e != cudaSuccess) return cuda_fail(e);
@@ -303,6 +305,29 @@ STREAMOPS_BINARY(stream_triad_f64, OP_TRIAD, double, DT_F64)
 STREAMOPS_BINARY(stream_triad_f32, OP_TRIAD, float, DT_F32)
 STREAMOPS_BINARY(stream_dot_f64, OP_DOT, double, DT_F64)
 STREAMOPS_BINARY(stream_dot_f32, OP_DOT, float, DT_F32)
+
+int stream_dot_wide_f32(const float *x, const float *y, double *out, double scalar, size_t n, streamops_stream_t stream) {
+    return run_op(OP_DOT, DT_F32, x, y, out, scalar, n, stream, true);
+}
+
+static int fold(int dtype, const double *partials, void *out, size_t count, streamops_stream_t stream) {
+    if (!out || (count > 0 && !partials)) return STREAMOPS_ERR_NULL;
+    if (((uintptr_t)partials % 8) || ((uintptr_t)out % (dtype == DT_F64 ? 8 : 4))) return STREAMOPS_ERR_ALIGN;
+    if (count > ((size_t)1 << 24)) return STREAMOPS_ERR_ARG;
+    if (count > 0 && ranges_overlap(partials, count * 8, out, dtype == DT_F64 ? 8 : 4)) return STREAMOPS_ERR_OVERLAP;
+    cudaError_t e = launch_fold(dtype, partials, count, out, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_launches.fetch_add(1);
+    return STREAMOPS_OK;
+}
+int stream_fold_f64(const double *partials, double *out, double scalar, size_t count, streamops_stream_t stream) {
+    (void)scalar;
+    return fold(DT_F64, partials, out, count, stream);
+}
+int stream_fold_f32(const double *partials, float *out, double scalar, size_t count, streamops_stream_t stream) {
+    (void)scalar;
+    return fold(DT_F32, partials, out, count, stream);
+}
 
 // Device-pointer chain: five asynchronous launches from one call.
 static int chain_device(int dtype, void *a, void *b, void *c, void *dot_out, double scalar, size_t n,

@@ -124,30 +124,52 @@ cudaError_t launch_pass1(const VecLaunch &c, const T *x, const T *y, size_t n, c
     return cudaGetLastError();
 }
 
+// Sequential left-to-right sum of count doubles by one thread: the order is the index order.
 template <typename T>
-cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, const T *x, const T *y, T *out, size_t n,
+__global__ void fold_kernel(const double *p, size_t count, T *out) {
+    double acc = 0.0;
+    for (size_t i = 0; i < count; ++i) acc += p[i];
+    out[0] = (T)acc;
+}
+
+template <typename T>
+cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, bool wide, const T *x, const T *y, void *out, size_t n,
                          const DotScratch &s, cudaStream_t st, int *launches) {
     if (c.grid > (unsigned)kMaxDotBlocks) return cudaErrorInvalidValue;
+    if (wide) {                       // the unrounded double total: pass 1 as usual, pass 2 writes a double
+        *launches = 2;
+        cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, (T *)nullptr, st);
+        if (e != cudaSuccess) return e;
+        dot_pass2_kernel<double><<<1, 1024, 0, st>>>(s.partials, c.grid, (double *)out);
+        return cudaGetLastError();
+    }
+    T *o = (T *)out;
     if (!two_pass) {
         *launches = 1;
-        return launch_pass1<T, true>(c, x, y, n, s, out, st);
+        return launch_pass1<T, true>(c, x, y, n, s, o, st);
     }
     *launches = 2;
-    cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, out, st);
+    cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, o, st);
     if (e != cudaSuccess) return e;
-    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, out);
+    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, o);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, const void *x, const void *y,
+cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, bool wide, const void *x, const void *y,
                        void *out, size_t n, const DotScratch &scratch, cudaStream_t stream, int *launches) {
     if (dtype == DT_F64)
-        return launch_dot_t<double>(cfg, two_pass, (const double *)x, (const double *)y, (double *)out, n,
+        return launch_dot_t<double>(cfg, two_pass, wide, (const double *)x, (const double *)y, out, n,
                                     scratch, stream, launches);
-    return launch_dot_t<float>(cfg, two_pass, (const float *)x, (const float *)y, (float *)out, n,
+    return launch_dot_t<float>(cfg, two_pass, wide, (const float *)x, (const float *)y, out, n,
                                scratch, stream, launches);
+}
+
+cudaError_t launch_fold(int dtype, const double *partials, size_t count, void *out, cudaStream_t stream) {
+    if (dtype == DT_F64) fold_kernel<double><<<1, 1, 0, stream>>>(partials, count, (double *)out);
+    else fold_kernel<float><<<1, 1, 0, stream>>>(partials, count, (float *)out);
+    return cudaGetLastError();
 }
 
 }  // namespace streamops

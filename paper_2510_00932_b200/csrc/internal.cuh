@@ -78,9 +78,12 @@ void note_launches(int n);              // adds to streamops_launch_count
 cudaError_t launch_elementwise(int op, int dtype, const VecLaunch &cfg, const void *x, const void *y,
                                void *out, double scalar, size_t n, cudaStream_t stream);
 // dot.cu
-cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, const void *x, const void *y,
+// `wide`: out is a double that receives the unrounded total, whatever the element type
+cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, bool wide, const void *x, const void *y,
                        void *out, size_t n, const DotScratch &scratch, cudaStream_t stream,
                        int *launches);
+// out[0] = (T)(((p[0] + p[1]) + p[2]) + ...), one thread, index order
+cudaError_t launch_fold(int dtype, const double *partials, size_t count, void *out, cudaStream_t stream);
 // bulk.cu
 cudaError_t launch_bulk(int op, int dtype, const BulkLaunch &cfg, const void *x, const void *y,
                         void *out, double scalar, size_t n, const DotScratch &scratch,

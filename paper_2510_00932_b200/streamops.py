@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
             f.argtypes, f.restype = [vp, vp, vp, dbl, sz, vp], ci
             f = getattr(L, f"streamops_chain_{t}")
             f.argtypes, f.restype = [vp, vp, vp, vp, dbl, sz, vp], ci
+        L.stream_dot_wide_f32.argtypes, L.stream_dot_wide_f32.restype = [vp, vp, vp, dbl, sz, vp], ci
+        for t in ("f32", "f64"):
+            f = getattr(L, f"stream_fold_{t}")
+            f.argtypes, f.restype = [vp, vp, dbl, sz, vp], ci
         L.stream_dot_noalloc_f64.argtypes, L.stream_dot_noalloc_f64.restype = [vp, vp, vp, dbl, sz, vp], ci
         L.shmem_mix_u32.argtypes, L.shmem_mix_u32.restype = [vp, vp, ctypes.c_uint, sz, vp], ci
         L.streamops_set_shmem_width.argtypes, L.streamops_set_shmem_width.restype = [ci], ci
@@ -168,6 +172,30 @@ def dot(x, y, out, scalar: float = 0.0):
     if x.numel() != y.numel() or out.numel() != 1:
         raise ValueError("dot takes two equal-length inputs and a one-element output")
     _raise(getattr(lib(), f"stream_dot_{suf}")(x.data_ptr(), y.data_ptr(), out.data_ptr(), float(scalar), x.numel(), stream))
+    return out
+
+
+def dot_wide(x, y, out64):
+    """out64[0] = the double-precision sum of x[i]*y[i] before any rounding to the element type;
+    out64 is a one-element float64 device tensor (stream_dot_wide_f32 / stream_dot_f64)."""
+    import torch
+    suf, stream = _marshal(x, y)
+    if x.numel() != y.numel() or out64.numel() != 1 or out64.dtype != torch.float64 or not out64.is_cuda:
+        raise ValueError("dot_wide takes two equal-length inputs and a one-element float64 device output")
+    f = lib().stream_dot_f64 if suf == "f64" else lib().stream_dot_wide_f32
+    _raise(f(x.data_ptr(), y.data_ptr(), out64.data_ptr(), 0.0, x.numel(), stream))
+    return out64
+
+
+def fold(partials, out):
+    """out[0] = the float64 partials added left to right, rounded once to out's type (stream_fold_*)."""
+    import torch
+    if partials.dtype != torch.float64 or not partials.is_cuda or not partials.is_contiguous() or partials.dim() != 1:
+        raise ValueError("fold takes a contiguous 1-D float64 device tensor of partial sums")
+    suf, stream = _marshal(out)
+    if out.numel() != 1:
+        raise ValueError("fold writes one element")
+    _raise(getattr(lib(), f"stream_fold_{suf}")(partials.data_ptr(), out.data_ptr(), 0.0, partials.numel(), stream))
     return out
 
 

@@ -153,3 +153,22 @@ def test_dot_abs_is_the_sum_of_magnitudes(oracle):
     xf, yf = x.astype(np.float32), y.astype(np.float32)
     truthf = sum(abs(Fraction(float(u)) * Fraction(float(v))) for u, v in zip(xf, yf))
     assert abs(Fraction(oracle.dot_abs(xf, yf)) - truthf) <= Fraction(1e-15) * truthf
+
+
+def test_fold_adds_left_to_right_with_one_rounding_per_step(oracle):
+    """The fold of per-GPU partial sums is pinned by inputs on which every other order, and any
+    wider accumulator, gives a different double."""
+    from fractions import Fraction
+    from oracle import exact
+    f = lambda *v: oracle.fold(np.array(v, dtype=np.float64))
+    assert f() == 0.0 and f(3.5) == 3.5
+    assert f(1e16, 1.0, -1e16) == 0.0                   # right-to-left or exact summation gives 1
+    assert f(-1e16, 1e16, 1.0) == 1.0
+    assert f(2.0 ** 53, 1.0, 1.0) == 2.0 ** 53          # pairwise (1 + 1 first) gives 2^53 + 2
+    assert f(1.0, 1.0, 2.0 ** 53) == 2.0 ** 53 + 2.0
+    rng = np.random.Generator(np.random.PCG64(77))
+    p = rng.standard_normal(64) * np.exp(rng.uniform(-30, 30, 64))
+    acc = Fraction(0)
+    for v in p:                                          # exact rational step, rounded to double every time
+        acc = Fraction(exact.round_to_format(acc + Fraction(float(v)), "f64"))
+    assert oracle.fold(p) == float(acc)
