@@ -96,9 +96,11 @@ shmem_mix_kernel(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n) {
 #pragma unroll
         for (int k = 0; k < kRows; ++k) stg_piece<VW>(dst + k * kCols, row[k]);
     }
-    // ragged tail: every word is a row of its own, doubled once per round, through shared memory too
+    // ragged tail: every word is a row of its own, doubled once per round, through shared memory too.
+    // The staging word is the first word of the thread's OWN piece of row 0: other warps of this
+    // block may still be working on their pieces of the last tile, and there is no barrier.
     if (blockIdx.x == (unsigned)(tiles % gridDim.x)) {
-        const uint32_t slot = (uint32_t)__cvta_generic_to_shared(tile) + threadIdx.x * 4;
+        const uint32_t slot = mine;
         for (size_t i = tiles * kTileWords + threadIdx.x; i < n; i += TH) {
             Piece<1> w;
             w.w[0] = x[i];

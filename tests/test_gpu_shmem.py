@@ -82,6 +82,22 @@ def test_in_place_and_more_tiles_than_blocks(so, torch, oracle):
     _check(torch, fx, dx, oracle.shmem_mix(x, 5, nthreads=len(os.sched_getaffinity(0))), 0)
 
 
+def test_tail_block_still_busy_with_its_last_tile(so, torch, oracle):
+    # the block that owns the ragged tail also owns tiles; its warps reach the tail at different times
+    so.set_shmem_width(16)
+    for tiles, tail, rounds in ((2220 + 280, 8191, 64), (741, 4097, 200), (3, 5000, 300)):
+        n = tiles * TILE + tail
+        x = inputs.make_words(n, seed=24)
+        want = oracle.shmem_mix(x, rounds, nthreads=len(os.sched_getaffinity(0)))
+        dx = torch.from_numpy(x.view(np.int32)).cuda()
+        do = torch.empty_like(dx)
+        for _ in range(4):
+            do.zero_()
+            so.shmem_mix(dx, do, rounds)
+            torch.cuda.synchronize()
+            assert (do.cpu().numpy().view(np.uint32) == want).all()
+
+
 def test_benchmark_size_and_paper_default_repetitions(so, torch, oracle):
     so.set_shmem_width(16)
     n, rounds = 1 << 24, 600                              # the configuration bench.py times
