@@ -132,13 +132,17 @@ int streamops_chain_f64(double *a, double *b, double *c, double *dot_out, double
 int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double scalar, size_t n, streamops_stream_t stream);
 
 /* One pass of the five kernels over three HOST arrays of n elements each, in the textbook
- * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The three arrays are
- * copied to the device, the five kernels above run on them, and the three arrays and the dot
- * product are copied back; the call returns after the results are in host memory. a, b, c and
- * dot_out are HOST pointers owned by the caller (pinned memory makes the copies asynchronous to
- * each other; pageable memory works). Device buffers are allocated on the first call and reused
- * while n does not grow; streamops_shutdown frees them. This is the end-to-end entry point for
- * callers whose data lives on the host. */
+ * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The arrays are cut into pieces
+ * of 16 MiB per array; each piece is copied to the device, run through the five kernels and copied
+ * back on three streams of the library's own, so that uploads, kernels and downloads of different
+ * pieces overlap and both directions of the host link are in use at once; the call returns after
+ * all results are in host memory. The dot product is the left-to-right sum of the pieces' double-
+ * precision partial dot products, rounded once: a fixed function of n, repeatable bit for bit, and
+ * within the same tolerance as stream_dot_* (not bitwise equal to it). a, b, c and dot_out are HOST
+ * pointers owned by the caller (pinned memory lets the copies overlap; pageable memory works).
+ * Device buffers are allocated on the first call and reused while n does not grow;
+ * streamops_shutdown frees them. This is the end-to-end entry point for callers whose data lives
+ * on the host. */
 int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out);
 int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out);
 

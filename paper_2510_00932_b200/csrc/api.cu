@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "../../include/streamops.h"
 #include "internal.cuh"
@@ -23,8 +24,10 @@ struct DeviceState {
     // host-path buffers (streamops_chain_host_*)
     void *chain_buf[3] = {nullptr, nullptr, nullptr};
     void *chain_dot = nullptr;
+    double *chain_partials = nullptr;                  // one double per piece
     size_t chain_bytes = 0;
-    cudaStream_t chain_stream = nullptr;
+    cudaStream_t chain_streams[3] = {nullptr, nullptr, nullptr};   // upload, kernels, download
+    std::vector<cudaEvent_t> chain_events;
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -242,6 +245,14 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
     return STREAMOPS_OK;
 }
 
+// Host-buffer pass, pipelined: the arrays are cut into pieces of kChainPieceBytes per array; piece k
+// is uploaded on one stream, run through the five kernels on a second (Dot as a double partial sum
+// per piece), and downloaded on a third, so that uploads, kernels and downloads of different pieces
+// overlap and the two directions of the host link are busy at the same time. The dot product is the
+// left-to-right fold of the per-piece partial sums: fixed by n alone, so repeatable bit for bit.
+constexpr size_t kChainPieceBytes = (size_t)16 << 20;
+constexpr size_t kChainMaxPieces = 4096;
+
 template <typename T>
 int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
     constexpr int dtype = sizeof(T) == 8 ? DT_F64 : DT_F32;
@@ -252,9 +263,13 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
     std::lock_guard<std::mutex> lock(g_mutex);
     cudaError_t e;
     const size_t bytes = n * sizeof(T);
-    if (!d->chain_stream && (e = cudaStreamCreateWithFlags(&d->chain_stream, cudaStreamNonBlocking)) != cudaSuccess)
-        return cuda_fail(e);
-    if (!d->chain_dot && cudaMalloc(&d->chain_dot, 8) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_ERR_WORKSPACE; }
+    for (cudaStream_t &st : d->chain_streams)
+        if (!st && (e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+    if (!d->chain_dot && (cudaMalloc(&d->chain_dot, 8) != cudaSuccess ||
+                          cudaMalloc(&d->chain_partials, sizeof(double) * kChainMaxPieces) != cudaSuccess)) {
+        (void)cudaGetLastError();
+        return STREAMOPS_ERR_WORKSPACE;
+    }
     if (bytes > d->chain_bytes) {
         for (void *&p : d->chain_buf) { cudaFree(p); p = nullptr; }
         d->chain_bytes = 0;
@@ -262,22 +277,43 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
             if (cudaMalloc(&p, bytes) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_ERR_WORKSPACE; }
         d->chain_bytes = bytes;
     }
-    cudaStream_t st = d->chain_stream;
-    T *da = (T *)d->chain_buf[0], *db = (T *)d->chain_buf[1], *dc = (T *)d->chain_buf[2], *dd = (T *)d->chain_dot;
+    // pieces: whole multiples of 32 bytes, at most kChainMaxPieces of them
+    size_t piece = kChainPieceBytes / sizeof(T);
+    while ((n + piece - 1) / piece > kChainMaxPieces) piece *= 2;
+    const size_t pieces = n ? (n + piece - 1) / piece : 0;
+    while (d->chain_events.size() < 2 * pieces) {
+        cudaEvent_t ev;
+        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        d->chain_events.push_back(ev);
+    }
+    cudaStream_t up = d->chain_streams[0], run = d->chain_streams[1], down = d->chain_streams[2];
     T *host[3] = {a, b, c};
-    T *dev[3] = {da, db, dc};
-    for (int i = 0; i < 3 && n > 0; ++i)
-        if ((e = cudaMemcpyAsync(dev[i], host[i], bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-    // c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b)
-    if ((status = run_op(OP_COPY, dtype, da, nullptr, dc, scalar, n, st)) != STREAMOPS_OK) return status;
-    if ((status = run_op(OP_SCALE, dtype, dc, nullptr, db, scalar, n, st)) != STREAMOPS_OK) return status;
-    if ((status = run_op(OP_ADD, dtype, da, db, dc, scalar, n, st)) != STREAMOPS_OK) return status;
-    if ((status = run_op(OP_TRIAD, dtype, db, dc, da, scalar, n, st)) != STREAMOPS_OK) return status;
-    if ((status = run_op(OP_DOT, dtype, da, db, dd, scalar, n, st)) != STREAMOPS_OK) return status;
-    for (int i = 0; i < 3 && n > 0; ++i)
-        if ((e = cudaMemcpyAsync(host[i], dev[i], bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(dot_out, dd, sizeof(T), cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
+    T *dev[3] = {(T *)d->chain_buf[0], (T *)d->chain_buf[1], (T *)d->chain_buf[2]};
+    T *dd = (T *)d->chain_dot;
+    for (size_t k = 0; k < pieces; ++k) {
+        const size_t lo = k * piece, len = n - lo < piece ? n - lo : piece;
+        cudaEvent_t uploaded = d->chain_events[2 * k], computed = d->chain_events[2 * k + 1];
+        for (int i = 0; i < 3; ++i)
+            if ((e = cudaMemcpyAsync(dev[i] + lo, host[i] + lo, len * sizeof(T), cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(uploaded, up)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(run, uploaded, 0)) != cudaSuccess) return cuda_fail(e);
+        T *pa = dev[0] + lo, *pb = dev[1] + lo, *pc = dev[2] + lo;
+        // c <- a; b <- s*c; c <- a+b; a <- b+s*c; partial dot(a, b)
+        if ((status = run_op(OP_COPY, dtype, pa, nullptr, pc, scalar, len, run)) != STREAMOPS_OK) return status;
+        if ((status = run_op(OP_SCALE, dtype, pc, nullptr, pb, scalar, len, run)) != STREAMOPS_OK) return status;
+        if ((status = run_op(OP_ADD, dtype, pa, pb, pc, scalar, len, run)) != STREAMOPS_OK) return status;
+        if ((status = run_op(OP_TRIAD, dtype, pb, pc, pa, scalar, len, run)) != STREAMOPS_OK) return status;
+        if ((status = run_op(OP_DOT, dtype, pa, pb, d->chain_partials + k, scalar, len, run, dtype == DT_F32)) != STREAMOPS_OK) return status;
+        if ((e = cudaEventRecord(computed, run)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(down, computed, 0)) != cudaSuccess) return cuda_fail(e);
+        for (int i = 0; i < 3; ++i)
+            if ((e = cudaMemcpyAsync(host[i] + lo, dev[i] + lo, len * sizeof(T), cudaMemcpyDeviceToHost, down)) != cudaSuccess) return cuda_fail(e);
+    }
+    if ((e = launch_fold(dtype, d->chain_partials, pieces, dd, run)) != cudaSuccess) return cuda_fail(e);
+    g_launches.fetch_add(1);
+    if ((e = cudaMemcpyAsync(dot_out, dd, sizeof(T), cudaMemcpyDeviceToHost, run)) != cudaSuccess) return cuda_fail(e);
+    for (cudaStream_t st : d->chain_streams)
+        if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
     return STREAMOPS_OK;
 }
 
@@ -374,9 +410,12 @@ int streamops_shutdown(void) {
         cudaDeviceSynchronize();
         cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag); cudaFree(d.chain_dot);
         for (void *&p : d.chain_buf) { cudaFree(p); p = nullptr; }
-        if (d.chain_stream) cudaStreamDestroy(d.chain_stream);
+        cudaFree(d.chain_partials); d.chain_partials = nullptr;
+        for (cudaStream_t &st : d.chain_streams) { if (st) cudaStreamDestroy(st); st = nullptr; }
+        for (cudaEvent_t ev : d.chain_events) cudaEventDestroy(ev);
+        d.chain_events.clear();
         d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr; d.chain_dot = nullptr;
-        d.chain_stream = nullptr; d.chain_bytes = 0; d.ready = false;
+        d.chain_bytes = 0; d.ready = false;
     }
     cudaSetDevice(prev);
     return STREAMOPS_OK;

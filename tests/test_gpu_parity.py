@@ -284,15 +284,20 @@ def test_chain_on_the_small_configuration(so, torch, oracle, name):
         assert abs(dd.item() - od) <= DOT_TOL[w.dtype] * abs(od)
 
 
+@pytest.mark.parametrize("n", [(1 << 20) + 3, 5 * (1 << 22) + 77])     # one piece; several 16 MiB pieces and a ragged last one
 @pytest.mark.parametrize("t,scalar", [("f64", 0.4), ("f32", 3.0)])
-def test_host_entry_point(so, torch, oracle, t, scalar):
-    n = (1 << 20) + 3
+def test_host_entry_point(so, torch, oracle, t, scalar, n):
     a, b, c = (_data(t, n, s) for s in (61, 62, 63))
     ha, hb, hc = a.copy(), b.copy(), c.copy()
     d = so.chain_host(ha, hb, hc, scalar)
     oa, ob, oc, od = oracle.chain(a, b, c, scalar)
     assert_bits_equal(ha, oa, "a"); assert_bits_equal(hb, ob, "b"); assert_bits_equal(hc, oc, "c")
     assert abs(float(d) - od) <= DOT_TOL[t] * abs(od)
+    ha2, hb2, hc2 = a.copy(), b.copy(), c.copy()                        # pinned or not, first call or not: same bits
+    pin = [torch.from_numpy(v).pin_memory() for v in (ha2, hb2, hc2)]
+    d2 = so.chain_host(*(p.numpy() for p in pin), scalar)
+    assert np.array([d2]).tobytes() == np.array([d]).tobytes()
+    assert_bits_equal(pin[0].numpy(), oa, "a, pinned")
     assert so.chain_host(ha[:0], hb[:0], hc[:0], scalar) == 0
 
 
