@@ -181,7 +181,8 @@ typedef struct streamops_tuning {
     int vec_bytes;      /* kind 0: 16 or 32 (256-bit ld/st.global) */
     int unroll;         /* kind 0: vectors per thread per array in flight: 1, 2 or 4 */
     int threads;        /* threads per block: 128, 256 or 512 (kind 1: consumer threads) */
-    int blocks_per_sm;  /* persistent grid = blocks_per_sm * SMs; 0 = one block per tile */
+    int blocks_per_sm;  /* persistent grid = blocks_per_sm * SMs; 0 = one block per tile (Dot: 0 = 2 or 3 per
+                           SM, chosen from the number of tiles) */
     int policy;         /* kind 0 cache-hint set, 0..7 (see streamops_policy_name) */
     int contiguous;     /* 0 = tiles interleaved across blocks, 1 = one contiguous range per block */
     int chunk_bytes;    /* kind 1: bytes per bulk copy per array (multiple of 16, <= 65536) */
@@ -193,7 +194,7 @@ typedef struct streamops_tuning {
                            resident while the previous kernel of the stream drains, and wait inside
                            the kernel until it has completed (hides launch latency) */
     int keep_mib;       /* kind 0, policies 7 and 8: the last keep_mib MiB of output in traversal order are
-                           stored with normal (7) or evict_last (8) L2 priority and are what the kernel
+                           stored plainly (7) or with evict_last L2 priority (8) and are what the kernel
                            leaves in L2 for its consumer; everything before is stored evict_first, so that
                            the kernel's own output does not push out the lines its producer left there */
 } streamops_tuning_t;

@@ -57,10 +57,8 @@ streamops_tuning_t default_tuning(int op, int dtype) {
         case OP_SCALE: t.reverse = 1; break;
         case OP_ADD:   t.threads = 128; break;
         case OP_TRIAD: t.threads = 128; t.reverse = 1; break;
-        // Dot: a persistent grid of 3 blocks per SM. With the 512-thread blocks of the double kernel only
-        // 2 fit at a time: the third starts as others finish and evens out the tail (measured 1-2 %
-        // over 2 per SM); the float kernel does best with 256-thread blocks, all 3 resident
-        case OP_DOT:   t.threads = f64 ? 512 : 256; t.blocks_per_sm = 3; t.policy = 4; t.unroll = 4; break;
+        // Dot: persistent grid sized automatically (blocks_per_sm = 0: 2 or 3 per SM, see resolve_vec)
+        case OP_DOT:   t.threads = f64 ? 512 : 256; t.blocks_per_sm = 0; t.policy = 4; t.unroll = 4; break;
     }
     return t;
 }
@@ -174,6 +172,12 @@ VecLaunch resolve_vec(const streamops_tuning_t &t, const DeviceState &d, int op,
     const size_t per_tile = (size_t)c.threads * (c.vec_bytes ? (size_t)c.unroll * c.vec_bytes / esize : 1);
     const size_t tiles = (n + per_tile - 1) / per_tile;
     size_t grid = t.blocks_per_sm > 0 ? (size_t)t.blocks_per_sm * d.sm_count : tiles;
+    if (op == OP_DOT && t.blocks_per_sm == 0) {
+        // automatic persistent grid: a third block per SM (which starts as the first two finish and
+        // evens out the tail) pays once every block has several tiles; small arrays do best with two
+        const size_t three = (size_t)3 * d.sm_count;
+        grid = tiles >= 6 * three ? three : (size_t)2 * d.sm_count;
+    }
     if (grid > tiles) grid = tiles;                            // never more blocks than tiles
     if (op == OP_DOT && grid > (size_t)kMaxDotBlocks) grid = kMaxDotBlocks;
     c.grid = clamp_grid(grid);
@@ -451,7 +455,7 @@ const char *streamops_policy_name(int policy) {
         case 4: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first";
         case 5: return "ld.global.L1::no_allocate + L2 evict_first / st.global";
         case 6: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_last";
-        case 7: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, evict_normal for the last keep_mib MiB";
+        case 7: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, plain st.global for the last keep_mib MiB";
         case 8: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, evict_last for the last keep_mib MiB";
         default: return "unknown";
     }

@@ -71,7 +71,7 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int
     for (; tile < end; tile += step) {
         const size_t v0 = (reverse ? ntiles - 1 - tile : tile) * tile_vecs + threadIdx.x;
         // two-phase stores: the first hot_tiles tiles of the traversal leave L2 first
-        const uint64_t stpol = (POL >= 7 && tile >= hot_tiles) ? l2.st_late : l2.st;
+        const uint64_t stpol = (POL == 8 && tile >= hot_tiles) ? l2.st_late : l2.st;
         Vec<VB> xv[U], yv[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
@@ -80,9 +80,13 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int
             for (int u = 0; u < U; ++u) ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
         }
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            apply_vec<T, OP, VB>(xv[u], yv[u], s);
-            stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], stpol);
+        for (int u = 0; u < U; ++u) apply_vec<T, OP, VB>(xv[u], yv[u], s);
+        if (POL == 7 && tile >= hot_tiles) {       // second phase of policy 7: plain stores (uniform per tile)
+#pragma unroll
+            for (int u = 0; u < U; ++u) stg<0>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], 0);
+        } else {
+#pragma unroll
+            for (int u = 0; u < U; ++u) stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], stpol);
         }
     }
     // ragged end, by the block that is next in line for a tile

@@ -10,8 +10,8 @@
 //   5  loads as 4 (read-once data leaves L2 first), plain st.global (written data stays)
 //   6  loads as 4, stores with an L2 evict_last policy (written data is kept for the next kernel)
 //   7  loads as 4; stores in two phases: L2 evict_first while the kernel is still consuming what
-//      its predecessor left in L2 (its own output must not push those lines out), normal
-//      priority afterwards (so that the kernel's last-written lines are what it leaves behind)
+//      its predecessor left in L2 (its own output must not push those lines out), plain
+//      st.global afterwards (so that the kernel's last-written lines are what it leaves behind)
 //   8  as 7 with L2 evict_last in the second phase (the consumer's evict_first loads demote the
 //      lines again once they have been read)
 // 16-byte accesses are .v4.b32; 32-byte accesses are the 256-bit .v8.b32 form of sm_100.
@@ -32,11 +32,6 @@ __device__ __forceinline__ uint64_t make_evict_first_policy() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
-__device__ __forceinline__ uint64_t make_evict_normal_policy() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
 __device__ __forceinline__ uint64_t make_evict_last_policy() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -50,7 +45,6 @@ template <int POL> __device__ __forceinline__ L2Policies make_l2_policies() {
     if constexpr (POL >= 4) p.ld = make_evict_first_policy();
     if constexpr (POL == 4 || POL == 7 || POL == 8) p.st = p.ld;
     if constexpr (POL == 6) p.st = make_evict_last_policy();
-    if constexpr (POL == 7) p.st_late = make_evict_normal_policy();
     if constexpr (POL == 8) p.st_late = make_evict_last_policy();
     return p;
 }
