@@ -57,8 +57,9 @@ streamops_tuning_t default_tuning(int op, int dtype) {
         case OP_SCALE: t.reverse = 1; break;
         case OP_ADD:   t.threads = 128; break;
         case OP_TRIAD: t.threads = 128; t.reverse = 1; break;
-        // Dot: persistent grid sized automatically (blocks_per_sm = 0: 2 or 3 per SM, see resolve_vec)
-        case OP_DOT:   t.threads = f64 ? 512 : 256; t.blocks_per_sm = 0; t.policy = 4; t.unroll = 4; break;
+        // Dot, double: persistent grid sized automatically (blocks_per_sm = 0: 2 or 3 per SM, see
+        // resolve_vec); float: 2 per SM and two vectors in flight measured best from 16 MiB to 2 GiB
+        case OP_DOT:   t.threads = 512; t.policy = 4; t.unroll = f64 ? 4 : 2; t.blocks_per_sm = f64 ? 0 : 2; break;
     }
     return t;
 }
