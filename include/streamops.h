@@ -197,6 +197,10 @@ typedef struct streamops_tuning {
                            stored plainly (7) or with evict_last L2 priority (8) and are what the kernel
                            leaves in L2 for its consumer; everything before is stored evict_first, so that
                            the kernel's own output does not push out the lines its producer left there */
+    int compensated;    /* Dot, kind 0: 1 = carry every accumulator as a (sum, error) pair (two-sum and, for
+                           double inputs, an exact product split: the published Dot2 scheme): the result is
+                           as accurate as a sum done in about twice the working precision, for inputs whose
+                           dot product cancels heavily; ~10 double operations per element instead of one */
 } streamops_tuning_t;
 
 int streamops_set_tuning(int op, int dtype, const streamops_tuning_t *t);

@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libstreamops.so")
 SOURCES = ["api.cu", "elementwise.cu", "ew_copy.cu", "ew_scale.cu", "ew_add.cu", "ew_triad.cu",
-           "dot.cu", "bulk.cu", "dot_noalloc.cu", "shmem.cu"]
+           "dot.cu", "dot_comp.cu", "bulk.cu", "dot_noalloc.cu", "shmem.cu"]
 # -fmad=false is a second guard beside the explicit *_rn intrinsics; Dot asks for fma() by name.
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-Xcompiler", "-fPIC"]

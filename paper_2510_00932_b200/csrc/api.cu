@@ -50,7 +50,7 @@ std::atomic<unsigned long long> g_launches{0};
 streamops_tuning_t default_tuning(int op, int dtype) {
     streamops_tuning_t t;
     t.kind = 0; t.vec_bytes = 32; t.unroll = 2; t.threads = 256; t.blocks_per_sm = 0;
-    t.policy = 7; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0; t.reverse = 0; t.pdl = 1; t.keep_mib = 112;
+    t.policy = 7; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0; t.reverse = 0; t.pdl = 1; t.keep_mib = 112; t.compensated = 0;
     const bool f64 = dtype == DT_F64;
     switch (op) {
         case OP_COPY:  break;
@@ -195,6 +195,7 @@ bool valid_tuning(const streamops_tuning_t &t) {
     if (t.blocks_per_sm < 0 || t.blocks_per_sm > 32) return false;
     if (t.policy < 0 || t.policy > 8) return false;
     if (t.keep_mib < 0 || t.keep_mib > 65536) return false;
+    if (t.compensated != 0 && t.compensated != 1) return false;
     if (t.chunk_bytes < 1024 || t.chunk_bytes > 65536 || (t.chunk_bytes & 15)) return false;
     if (t.stages < 2 || t.stages > 8) return false;
     return true;
@@ -242,7 +243,12 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
         e = launch_bulk(op, dtype, b, x, y, out, scalar, n, scratch, d->error_flag, stream, &launches);
     } else {
         const VecLaunch c = resolve_vec(t, *d, op, esize, x, y, out, n);
-        if (op == OP_DOT) e = launch_dot(dtype, c, t.two_pass != 0, wide, x, y, out, n, scratch, stream, &launches);
+        if (op == OP_DOT && t.compensated && !wide) {
+            VecLaunch cc = c;
+            if (cc.vec_bytes != 32) cc.vec_bytes = 0;                    // 32-byte vectors or the scalar loop
+            if (cc.grid > (unsigned)kMaxDotBlocks / 2) cc.grid = kMaxDotBlocks / 2;
+            e = launch_dot_compensated(dtype, cc, x, y, out, n, scratch, stream);
+        } else if (op == OP_DOT) e = launch_dot(dtype, c, t.two_pass != 0, wide, x, y, out, n, scratch, stream, &launches);
         else e = launch_elementwise(op, dtype, c, x, y, out, scalar, n, stream);
     }
     if (e != cudaSuccess) return cuda_fail(e);

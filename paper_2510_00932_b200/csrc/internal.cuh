@@ -82,6 +82,9 @@ cudaError_t launch_elementwise(int op, int dtype, const VecLaunch &cfg, const vo
 cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, bool wide, const void *x, const void *y,
                        void *out, size_t n, const DotScratch &scratch, cudaStream_t stream,
                        int *launches);
+// dot_comp.cu: Dot with (sum, error) pairs throughout; one launch; cfg.grid <= kMaxDotBlocks / 2
+cudaError_t launch_dot_compensated(int dtype, const VecLaunch &cfg, const void *x, const void *y, void *out, size_t n,
+                                   const DotScratch &scratch, cudaStream_t stream);
 // out[0] = (T)(((p[0] + p[1]) + p[2]) + ...), one thread, index order
 cudaError_t launch_fold(int dtype, const double *partials, size_t count, void *out, cudaStream_t stream);
 // bulk.cu

@@ -117,3 +117,22 @@ def make_words(n: int, seed: int = 5) -> np.ndarray:
     """Uniform random 32-bit words for the shared-memory exchange microkernel (PCG64 stream)."""
     rng = np.random.Generator(np.random.PCG64(seed))
     return rng.integers(0, 1 << 32, size=int(n), dtype=np.uint32)
+
+
+def make_cancelling(n: int, dtype: str = "f64", seed: int = 6, log2_big: int = 40):
+    """Two arrays whose dot product cancels heavily: shuffled triples x = (A, r, -A), y = (B, s, B)
+    with |A*B| about 2**log2_big times |r*s|, so that the large products cancel in pairs and only
+    the sum of the r*s survives (condition number about 2**(log2_big + 1)). Values are random, no
+    arithmetic of the kernels under test is involved. n is rounded down to a multiple of 3."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    t = n // 3
+    np_t = np.float64 if dtype == "f64" else np.float32
+    half = log2_big // 2
+    A = (rng.uniform(1.0, 2.0, t) * 2.0 ** half).astype(np_t)
+    B = (rng.uniform(1.0, 2.0, t) * 2.0 ** (log2_big - half)).astype(np_t)
+    r = rng.uniform(-1.0, 1.0, t).astype(np_t)
+    s = rng.uniform(-1.0, 1.0, t).astype(np_t)
+    x = np.concatenate([A, r, -A])
+    y = np.concatenate([B, s, B])
+    perm = rng.permutation(3 * t)
+    return np.ascontiguousarray(x[perm]), np.ascontiguousarray(y[perm])
