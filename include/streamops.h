@@ -145,6 +145,9 @@ int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double sca
  * on the host. */
 int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out);
 int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out);
+/* Size of one piece of the host-buffer pipeline, per array, in MiB (1..4096; default 16). The dot
+ * product's last bits depend on it (the pieces' partial sums are folded in order). */
+int streamops_set_host_piece_mib(int mib);
 
 /* Shared-memory exchange microkernel. Table 1 of the paper lists a shared-memory benchmark whose one
  * parameter is a repetition count (300..1500, default 600) and whose time goes into shared-memory

@@ -256,12 +256,12 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
     return STREAMOPS_OK;
 }
 
-// Host-buffer pass, pipelined: the arrays are cut into pieces of kChainPieceBytes per array; piece k
+// Host-buffer pass, pipelined: the arrays are cut into pieces of g_chain_piece_bytes per array; piece k
 // is uploaded on one stream, run through the five kernels on a second (Dot as a double partial sum
 // per piece), and downloaded on a third, so that uploads, kernels and downloads of different pieces
 // overlap and the two directions of the host link are busy at the same time. The dot product is the
 // left-to-right fold of the per-piece partial sums: fixed by n alone, so repeatable bit for bit.
-constexpr size_t kChainPieceBytes = (size_t)16 << 20;
+std::atomic<size_t> g_chain_piece_bytes{(size_t)16 << 20};
 constexpr size_t kChainMaxPieces = 4096;
 
 template <typename T>
@@ -289,7 +289,7 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
         d->chain_bytes = bytes;
     }
     // pieces: whole multiples of 32 bytes, at most kChainMaxPieces of them
-    size_t piece = kChainPieceBytes / sizeof(T);
+    size_t piece = g_chain_piece_bytes.load() / sizeof(T);
     while ((n + piece - 1) / piece > kChainMaxPieces) piece *= 2;
     const size_t pieces = n ? (n + piece - 1) / piece : 0;
     while (d->chain_events.size() < 2 * pieces) {
@@ -403,6 +403,12 @@ int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, siz
 }
 int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out) {
     return chain_host<float>(a, b, c, scalar, n, dot_out);
+}
+
+int streamops_set_host_piece_mib(int mib) {
+    if (mib < 1 || mib > 4096) return STREAMOPS_ERR_ARG;
+    g_chain_piece_bytes.store((size_t)mib << 20);
+    return STREAMOPS_OK;
 }
 
 int streamops_init(int device) {

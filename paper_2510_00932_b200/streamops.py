@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.streamops_set_shmem_width.argtypes, L.streamops_set_shmem_width.restype = [ci], ci
         L.streamops_get_shmem_width.argtypes, L.streamops_get_shmem_width.restype = [], ci
         L.streamops_init.argtypes, L.streamops_init.restype = [ci], ci
+        L.streamops_set_host_piece_mib.argtypes, L.streamops_set_host_piece_mib.restype = [ci], ci
         L.streamops_shutdown.argtypes, L.streamops_shutdown.restype = [], ci
         L.streamops_set_tuning.argtypes, L.streamops_set_tuning.restype = [ci, ci, ctypes.POINTER(Tuning)], ci
         L.streamops_get_tuning.argtypes, L.streamops_get_tuning.restype = [ci, ci, ctypes.POINTER(Tuning)], ci
@@ -261,6 +262,10 @@ def chain_host(a, b, c, scalar: float):
     _raise(getattr(lib(), f"streamops_chain_host_{suf}")(a.ctypes.data, b.ctypes.data, c.ctypes.data,
                                                         float(scalar), a.size, res.ctypes.data))
     return res[0]
+
+
+def set_host_piece_mib(mib: int):
+    _raise(lib().streamops_set_host_piece_mib(int(mib)))
 
 
 def init(device: int = 0):

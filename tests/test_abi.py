@@ -53,6 +53,12 @@ def test_tuning_table_validation_needs_no_gpu(so):
     assert so.get_tuning("triad", "f64").unroll == t.unroll
 
 
+def test_host_piece_size_validation(so):
+    L = so.lib()
+    assert L.streamops_set_host_piece_mib(0) == 7 and L.streamops_set_host_piece_mib(5000) == 7
+    assert L.streamops_set_host_piece_mib(16) == 0
+
+
 def test_binding_rejects_host_tensors(so):
     import torch
     x = torch.zeros(8, dtype=torch.float64)
