@@ -33,10 +33,10 @@ UNIT = "GB/s"
 NCU_TRAFFIC_BYTES: dict = {
     # profiles/ncu_chain_dram_c2_fp64.md (L2 state kept between kernels, as in the timed loop):
     # add reads 465.9 MB + writes 272.9 MB; triad reads 464.1 MB + writes 266.6 MB per launch
-    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "keep_mib": 112, "kind": 0, "pdl": 1, '
-                  '"policy": 7, "reverse": 0, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 738_800_000,
-    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "contiguous": 0, "keep_mib": 112, "kind": 0, "pdl": 1, '
-                    '"policy": 7, "reverse": 1, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 730_700_000,
+    ("c2", "add", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "compensated": 0, "contiguous": 0, "keep_mib": 112, "kind": 0, "pdl": 1, '
+                  '"policy": 7, "reverse": 2, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 738_800_000,
+    ("c2", "triad", '{"blocks_per_sm": 0, "chunk_bytes": 16384, "compensated": 0, "contiguous": 0, "keep_mib": 112, "kind": 0, "pdl": 1, '
+                    '"policy": 7, "reverse": 2, "stages": 4, "threads": 128, "two_pass": 0, "unroll": 2, "vec_bytes": 32}'): 730_700_000,
 }
 
 

@@ -191,8 +191,11 @@ typedef struct streamops_tuning {
     int chunk_bytes;    /* kind 1: bytes per bulk copy per array (multiple of 16, <= 65536) */
     int stages;         /* kind 1: ring depth, 2..8 */
     int two_pass;       /* Dot only: 1 = second pass as its own launch, 0 = last block finishes */
-    int reverse;        /* kind 0: 1 = walk the array from its end to its start (L2 reuse when the
-                           previous kernel wrote this kernel's input front to back) */
+    int reverse;        /* kind 0: 0 = walk the arrays from start to end, 1 = from end to start, 2 = automatic
+                           (elementwise kernels; the default): from the end IF an input of this call is the
+                           array the previous elementwise call on this device wrote and that call finished
+                           at the high end, so that the lines it left in L2 are read first. Results do not
+                           depend on the direction; Dot treats 2 as 0 (its summation order is fixed) */
     int pdl;            /* kind 0: 1 = programmatic dependent launch: the kernel's blocks may become
                            resident while the previous kernel of the stream drains, and wait inside
                            the kernel until it has completed (hides launch latency) */

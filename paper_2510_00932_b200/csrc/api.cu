@@ -21,6 +21,12 @@ struct DeviceState {
     unsigned *tickets = nullptr;       // kDotSlots counters, zero between calls
     int *error_flag = nullptr;         // set by a bounded wait that gave up
     std::atomic<unsigned> next_slot{0};
+    // the array most recently written by an elementwise kernel on this device and the end of it that
+    // was written last (1 = high addresses): where its still-cached lines are. Packed into atomics;
+    // a stale or torn reading only costs bandwidth.
+    std::atomic<uintptr_t> last_written{0};
+    std::atomic<size_t> last_written_bytes{0};
+    std::atomic<int> last_written_end_high{0};
     // host-path buffers (streamops_chain_host_*)
     void *chain_buf[3] = {nullptr, nullptr, nullptr};
     void *chain_dot = nullptr;
@@ -38,10 +44,11 @@ std::atomic<unsigned long long> g_launches{0};
 // Defaults: the measured best launch shapes on B200 for arrays far larger than L2 (fp64 n = 2^25,
 // fp32 n = 2^26). The elementwise kernels run one block per tile: the hardware block scheduler
 // then balances the two dies' unequal distance to memory better than a static persistent grid.
-// L2 use across consecutive kernels: loads are marked evict-first (read-once data), and scale and
-// triad walk their arrays from the end, so that in the sequence copy, scale, add, triad, dot every
-// kernel starts where its producer stopped and finds the producer's last-written lines still in
-// L2. Stores are two-phase: evict-first while the kernel is still reading those inherited lines
+// L2 use across consecutive kernels: loads are marked evict-first (read-once data), and a kernel that
+// reads the array the previous kernel wrote walks it from the end that kernel wrote last (reverse = 2,
+// automatic): in the sequence copy, scale, add, triad, dot that makes scale and triad walk backwards,
+// and every kernel starts where its producer stopped and finds the producer's last-written lines
+// still in L2. Stores are two-phase: evict-first while the kernel is still reading those inherited lines
 // (its own output would otherwise push them out), normal priority for the last 112 MiB it writes,
 // which is what it leaves behind for its consumer (measured at fp64 n = 2^25: 337 MB, 16 %, fewer
 // DRAM reads per pass of the five kernels than with no reuse; 297 MB with one-phase stores).
@@ -53,10 +60,10 @@ streamops_tuning_t default_tuning(int op, int dtype) {
     t.policy = 7; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0; t.reverse = 0; t.pdl = 1; t.keep_mib = 112; t.compensated = 0;
     const bool f64 = dtype == DT_F64;
     switch (op) {
-        case OP_COPY:  break;
-        case OP_SCALE: t.reverse = 1; break;
-        case OP_ADD:   t.threads = 128; break;
-        case OP_TRIAD: t.threads = 128; t.reverse = 1; break;
+        case OP_COPY:  t.reverse = 2; break;
+        case OP_SCALE: t.reverse = 2; break;
+        case OP_ADD:   t.threads = 128; t.reverse = 2; break;
+        case OP_TRIAD: t.threads = 128; t.reverse = 2; break;
         // Dot, double: persistent grid sized automatically (blocks_per_sm = 0: 2 or 3 per SM, see
         // resolve_vec); float: 2 per SM and two vectors in flight measured best from 16 MiB to 2 GiB
         case OP_DOT:   t.threads = 512; t.policy = 4; t.unroll = f64 ? 4 : 2; t.blocks_per_sm = f64 ? 0 : 2; break;
@@ -164,7 +171,7 @@ VecLaunch resolve_vec(const streamops_tuning_t &t, const DeviceState &d, int op,
     c.unroll = t.unroll;
     c.threads = t.threads;
     c.contiguous = t.contiguous;
-    c.reverse = t.reverse != 0;
+    c.reverse = t.reverse == 1;                                  // 2 (automatic) is resolved by the caller
     c.pdl = t.pdl != 0;
     c.policy = t.policy;
     // the read-only data path must not be used on an array the kernel also writes
@@ -198,6 +205,7 @@ bool valid_tuning(const streamops_tuning_t &t) {
     if (t.compensated != 0 && t.compensated != 1) return false;
     if (t.chunk_bytes < 1024 || t.chunk_bytes > 65536 || (t.chunk_bytes & 15)) return false;
     if (t.stages < 2 || t.stages > 8) return false;
+    if (t.reverse < 0 || t.reverse > 2) return false;
     return true;
 }
 
@@ -242,7 +250,20 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
         b.grid = clamp_grid(grid);
         e = launch_bulk(op, dtype, b, x, y, out, scalar, n, scratch, d->error_flag, stream, &launches);
     } else {
-        const VecLaunch c = resolve_vec(t, *d, op, esize, x, y, out, n);
+        VecLaunch c = resolve_vec(t, *d, op, esize, x, y, out, n);
+        if (op != OP_DOT) {
+            if (t.reverse == 2) {
+                // automatic direction: if an input is the array the previous elementwise kernel wrote,
+                // start at the end that kernel wrote last (its lines are the ones still in L2)
+                const uintptr_t w = d->last_written.load();
+                const bool consumer = w != 0 && d->last_written_bytes.load() == n * esize &&
+                                      (w == (uintptr_t)x || (uses_y && w == (uintptr_t)y));
+                c.reverse = consumer && d->last_written_end_high.load() != 0;
+            }
+            d->last_written.store((uintptr_t)out);
+            d->last_written_bytes.store(n * esize);
+            d->last_written_end_high.store(c.reverse ? 0 : 1);       // a forward walk finishes at the high end
+        }
         if (op == OP_DOT && t.compensated && !wide) {
             VecLaunch cc = c;
             if (cc.vec_bytes != 32) cc.vec_bytes = 0;                    // 32-byte vectors or the scalar loop
