@@ -186,8 +186,8 @@ SHMEM_TILE = SHMEM_ROWS * SHMEM_COLS
 
 def shmem_mix(x: np.ndarray, rounds: int, nthreads: int = 1) -> np.ndarray:
     """Shared-memory exchange microkernel (the definition is in shmem_oracle.c): tiles of 8 rows
-    x 1024 columns of 32-bit words; a round adds to every row the row below it (cyclically, modulo
-    2^32); words past the last whole tile double every round. ``nthreads`` > 1 only deals whole
+    x 1024 columns of 32-bit words; a round adds to every row the two rows below it (cyclically,
+    modulo 2^32); words past the last whole tile triple every round. ``nthreads`` > 1 only deals whole
     tiles to threads."""
     if not (isinstance(x, np.ndarray) and x.dtype == np.uint32 and x.ndim == 1 and x.flags.c_contiguous):
         raise ValueError("shmem_mix takes a contiguous 1-D uint32 array")

@@ -19,7 +19,7 @@ import oracle                                                     # noqa: E402
 from paper_2510_00932_b200 import inputs                          # noqa: E402
 
 CASES = [("c1", None), ("c2", 1 << 22), ("c3", 1 << 22), ("c4", 1 << 22)]     # (workload, length override)
-SHMEM = [((1 << 20) + 77, 600), (3 * 8192 + 5, 7)]
+SHMEM = [((1 << 20) + 77, 600), ((1 << 18) + 4099, 1500), (3 * 8192 + 5, 7)]
 
 
 def compute():
