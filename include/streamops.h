@@ -153,10 +153,13 @@ int streamops_set_host_piece_mib(int mib);
  * parameter is a repetition count (300..1500, default 600) and whose time goes into shared-memory
  * loads and stores (Table 2); the paper does not define it, so the operation is this library's own:
  *   the n 32-bit words of x are cut into tiles of 8 rows x 1024 columns (row-major, 8192 words);
- *   one round replaces, in every tile, row k by row k + row ((k + 1) mod 8), all eight rows taken
- *   from the values before the round, addition modulo 2^32; a word past the last whole tile is a
- *   row of its own and is doubled by a round; out = the array after `rounds` rounds.
- * (Equivalently row k of the result is sum_j C(rounds, j) * row (k + j) mod 8.) Every round moves
+ *   one round replaces, in every tile, row k by row k + row ((k + 1) mod 8) + row ((k + 2) mod 8),
+ *   all eight rows taken from the values before the round, addition modulo 2^32; a word past the
+ *   last whole tile is a one-row tile of its own and is tripled by a round; out = the array after
+ *   `rounds` rounds.
+ * (Equivalently row k of the result is sum_j w_j * row (k + j) mod 8, w_j the sum of the coefficients
+ * of x^m, m = j mod 8, in (1 + x + x^2)^rounds. The round is a bijection, so the output depends on
+ * every input word and on `rounds` however many rounds are run.) Every round moves
  * each word through shared memory once in each direction: 8 * rounds bytes of shared-memory
  * traffic per word against 8 bytes of global traffic, so for rounds >> 5 the kernel is bound by
  * shared-memory bandwidth (128 bytes per clock per SM).

@@ -4,13 +4,15 @@
 // this library's own.
 //
 //   The n 32-bit words are cut into tiles of 8 rows x 1024 columns (row-major, 32 KiB). One round
-//   replaces row k by row k + row (k + 1) mod 8, all rows taken from before the round, modulo
-//   2^32. Words past the last whole tile are rows of their own: a round doubles them.
-//   out = the array after `rounds` rounds.
+//   replaces row k by row k + row (k + 1) mod 8 + row (k + 2) mod 8, all rows taken from before
+//   the round, modulo 2^32. A word past the last whole tile is a one-row tile of its own (its
+//   neighbours are itself): a round triples it. out = the array after `rounds` rounds.
+//   The round is a bijection (1 + x + x^2 is a unit modulo x^8 - 1 and 2^32; 3 is odd), so the
+//   result depends on every input word and on every round at any repetition count.
 //
 // A block stages a tile in shared memory; thread t owns VW adjacent columns, i.e. one 4*VW-byte
-// piece of every row, eight pieces in all. A round is eight shared-memory loads, the adds, and
-// eight shared-memory stores per thread; every value travels through shared memory every round
+// piece of every row, eight pieces in all. A round is eight shared-memory loads, one three-input
+// add per word, and eight shared-memory stores per thread; every value travels through shared memory every round
 // (the accesses are inline PTX, so the compiler cannot keep them in registers across rounds).
 // Pieces of one row are contiguous across the threads of a warp: no bank conflicts at any width.
 // No thread ever reads a column another thread writes, so there is no barrier in the loop --
@@ -82,11 +84,13 @@ shmem_mix_kernel(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n) {
         for (unsigned r = 0; r < rounds; ++r) {
 #pragma unroll
             for (int k = 0; k < kRows; ++k) lds<VW>(row[k], mine + k * kRowBytes);
-            const Piece<VW> first = row[0];
+            const Piece<VW> first = row[0], second = row[1];
 #pragma unroll
-            for (int k = 0; k < kRows; ++k) {
+            for (int k = 0; k < kRows; ++k) {           // ascending k: rows k + 1 and k + 2 still hold old values
 #pragma unroll
-                for (int e = 0; e < VW; ++e) row[k].w[e] += (k + 1 < kRows ? row[k + 1].w[e] : first.w[e]);
+                for (int e = 0; e < VW; ++e)
+                    row[k].w[e] += (k + 1 < kRows ? row[k + 1].w[e] : first.w[e]) +
+                                   (k + 2 < kRows ? row[k + 2].w[e] : (k + 2 == kRows ? first.w[e] : second.w[e]));
             }
 #pragma unroll
             for (int k = 0; k < kRows; ++k) sts<VW>(mine + k * kRowBytes, row[k]);
@@ -96,7 +100,7 @@ shmem_mix_kernel(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n) {
 #pragma unroll
         for (int k = 0; k < kRows; ++k) stg_piece<VW>(dst + k * kCols, row[k]);
     }
-    // ragged tail: every word is a row of its own, doubled once per round, through shared memory too.
+    // ragged tail: every word is a one-row tile of its own, tripled once per round, through shared memory too.
     // The staging word is the first word of the thread's OWN piece of row 0: other warps of this
     // block may still be working on their pieces of the last tile, and there is no barrier.
     if (blockIdx.x == (unsigned)(tiles % gridDim.x)) {
@@ -107,7 +111,7 @@ shmem_mix_kernel(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n) {
             sts<1>(slot, w);
             for (unsigned r = 0; r < rounds; ++r) {
                 lds<1>(w, slot);
-                w.w[0] += w.w[0];
+                w.w[0] += w.w[0] + w.w[0];
                 sts<1>(slot, w);
             }
             lds<1>(w, slot);

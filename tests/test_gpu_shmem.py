@@ -98,16 +98,22 @@ def test_tail_block_still_busy_with_its_last_tile(so, torch, oracle):
             assert (do.cpu().numpy().view(np.uint32) == want).all()
 
 
-def test_benchmark_size_and_paper_default_repetitions(so, torch, oracle):
+@pytest.mark.parametrize("rounds", [600, 1500])
+def test_benchmark_size_at_the_paper_default_and_largest_repetition_counts(so, torch, oracle, rounds):
     so.set_shmem_width(16)
-    n, rounds = 1 << 24, 600                              # the configuration bench.py times
+    n = (1 << 24) + 4099                                  # the benchmark's tile count plus a ragged tail
     x = inputs.make_words(n, seed=5)
     dx = torch.from_numpy(x.view(np.int32)).cuda()
     do = torch.empty_like(dx)
     so.shmem_mix(dx, do, rounds)
     torch.cuda.synchronize()
     want = oracle.shmem_mix(x, rounds, nthreads=len(os.sched_getaffinity(0)))
-    assert (do.cpu().numpy().view(np.uint32) == want).all()
+    got = do.cpu().numpy().view(np.uint32)
+    assert (got == want).all()
+    # the comparison is not one of zeros with zeros, and a kernel that stopped a round early fails it
+    assert inputs.checksum(want) != 0 and np.count_nonzero(want) > 0.99 * n
+    fewer = oracle.shmem_mix(x[:3 * TILE], rounds - 1)
+    assert (got[:3 * TILE] != fewer).mean() > 0.99
 
 
 def test_argument_errors(so, torch):
