@@ -43,7 +43,7 @@ enum streamops_status {
     STREAMOPS_ERR_ALIGN = 2,     /* a pointer not aligned to the element size */
     STREAMOPS_ERR_OVERLAP = 3,   /* out partially overlaps an input */
     STREAMOPS_ERR_CUDA = 4,      /* a CUDA call failed; see streamops_last_cuda_error */
-    STREAMOPS_ERR_WORKSPACE = 5, /* the per-device workspace could not be created */
+    STREAMOPS_ERR_WORKSPACE = 5, /* the per-device workspace could not be created, or every Dot slot is in flight */
     STREAMOPS_ERR_TIMEOUT = 6,   /* a bounded wait inside a bulk-copy kernel gave up */
     STREAMOPS_ERR_ARG = 7,       /* an argument outside its documented range */
     STREAMOPS_ERR_TOO_LARGE = 8  /* n exceeds what the fixed scratch of stream_dot_noalloc_f64 covers */
@@ -78,12 +78,25 @@ int stream_triad_f32(const float *x, const float *y, float *out, double scalar, 
  * summation order is a fixed function of n and the tuning in force -- never of block arrival
  * order or of the stream -- so repeated calls return identical bits. Accuracy: within relative
  * 1e-12 (double) / 1e-5 (float) of the exactly rounded dot product for the documented
- * workloads. Reads 2*n*sizeof(T) bytes. Uses one slot of the per-device workspace; at most
- * STREAMOPS_DOT_SLOTS Dot calls may be in flight on one device at a time (slots are handed out
- * round-robin; more concurrent calls than slots would share a slot and race). */
+ * workloads. Reads 2*n*sizeof(T) bytes.
+ * Workspace slots. Every Dot in flight needs a slot of the per-device workspace to itself. A stream
+ * keeps the slot it used last (its Dots run one after the other); a Dot on another stream takes a
+ * slot that was never used or whose last Dot has finished (the finishing kernel leaves a mark in
+ * device memory; when a slot has to change hands the call reads those marks with a small copy on a
+ * stream of the library's own and waits for that copy only, never for a caller's stream). When all
+ * STREAMOPS_DOT_SLOTS slots hold Dots still in flight on other streams the call launches nothing and
+ * returns STREAMOPS_ERR_WORKSPACE: wait for one of them and call again. It never shares a slot.
+ * Stream capture. A Dot issued while `stream` is being captured gets one of
+ * STREAMOPS_DOT_CAPTURE_SLOTS slots set aside for graphs (handed out in turn, never used by ordinary
+ * calls), and that slot is part of the captured launch: replays of one graph are safe against every
+ * ordinary call; two graphs replayed at the same time are safe against each other unless more than
+ * STREAMOPS_DOT_CAPTURE_SLOTS Dots have been captured in the process, after which slots repeat. A
+ * captured elementwise launch likewise keeps the traversal direction chosen at capture time (see
+ * `reverse` below); that affects speed only. */
 int stream_dot_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
 int stream_dot_f32(const float *x, const float *y, float *out, double scalar, size_t n, streamops_stream_t stream);
-#define STREAMOPS_DOT_SLOTS 32
+#define STREAMOPS_DOT_SLOTS 24
+#define STREAMOPS_DOT_CAPTURE_SLOTS 8
 
 /* The two pieces a Dot over an array that is split across GPUs is made of (the sum is the only step
  * of the five kernels that needs an exchange: one double per GPU).
@@ -116,7 +129,11 @@ int stream_fold_f32(const double *partials, float *out, double scalar, size_t co
  *     overlap in time on one GPU race on it and give wrong results: keep them on one stream or
  *     order them with events.
  *   - The first call on each device looks up the array's device address (once, with that device
- *     current). Make that first call outside stream capture.
+ *     current) and is the first launch from this part of the library, which makes the CUDA runtime
+ *     load the module that holds the kernel and the array: the driver reserves device memory for
+ *     them at that moment. So make one call per device at start-up -- outside stream capture, and
+ *     before the device's memory is handed to a pool that takes all of it; n = 1 is enough. Calls
+ *     after that first one leave the amount of free device memory unchanged.
  * The summation order differs from stream_dot_f64's, so the two agree to rounding, not bitwise. */
 int stream_dot_noalloc_f64(const double *x, const double *y, double *out, double scalar, size_t n, streamops_stream_t stream);
 #define STREAMOPS_DOT_NOALLOC_MAX_N (1ull << 28)
@@ -133,16 +150,18 @@ int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double sca
 
 /* One pass of the five kernels over three HOST arrays of n elements each, in the textbook
  * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The arrays are cut into pieces
- * of 16 MiB per array; each piece is copied to the device, run through the five kernels and copied
- * back on three streams of the library's own, so that uploads, kernels and downloads of different
- * pieces overlap and both directions of the host link are in use at once; the call returns after
- * all results are in host memory. The dot product is the left-to-right sum of the pieces' double-
+ * of 16 MiB per array; each piece is copied into a ring of four device stages (three piece buffers
+ * each: 192 MiB of device memory whatever n is, so the arrays may be far larger than the device's
+ * memory), run through the five kernels and copied back on three streams of the library's own, so
+ * that uploads, kernels and downloads of different pieces overlap and both directions of the host
+ * link are in use at once; the call returns after all results are in host memory. The dot product is the left-to-right sum of the pieces' double-
  * precision partial dot products, rounded once: a fixed function of n, repeatable bit for bit, and
  * within the same tolerance as stream_dot_* (not bitwise equal to it). a, b, c and dot_out are HOST
  * pointers owned by the caller (pinned memory lets the copies overlap; pageable memory works).
- * Device buffers are allocated on the first call and reused while n does not grow;
- * streamops_shutdown frees them. This is the end-to-end entry point for callers whose data lives
- * on the host. */
+ * The ring is allocated on the first call and reused while the piece size does not change;
+ * streamops_shutdown frees it. Calls from several threads on one device are serialised while they
+ * issue their work and wait only for their own results. This is the end-to-end entry point for
+ * callers whose data lives on the host. */
 int streamops_chain_host_f64(double *a, double *b, double *c, double scalar, size_t n, double *dot_out);
 int streamops_chain_host_f32(float *a, float *b, float *c, double scalar, size_t n, float *dot_out);
 /* Size of one piece of the host-buffer pipeline, per array, in MiB (1..4096; default 16). The dot
@@ -189,7 +208,7 @@ typedef struct streamops_tuning {
     int threads;        /* threads per block: 128, 256 or 512 (kind 1: consumer threads) */
     int blocks_per_sm;  /* persistent grid = blocks_per_sm * SMs; 0 = one block per tile (Dot: 0 = 2 or 3 per
                            SM, chosen from the number of tiles) */
-    int policy;         /* kind 0 cache-hint set, 0..7 (see streamops_policy_name) */
+    int policy;         /* kind 0 cache-hint set, 0..8 (see streamops_policy_name) */
     int contiguous;     /* 0 = tiles interleaved across blocks, 1 = one contiguous range per block */
     int chunk_bytes;    /* kind 1: bytes per bulk copy per array (multiple of 16, <= 65536) */
     int stages;         /* kind 1: ring depth, 2..8 */
@@ -220,6 +239,15 @@ const char *streamops_policy_name(int policy);
 /* Reads the device error flag of the current device (a bounded wait that gave up sets it),
  * after synchronising `stream`. Returns STREAMOPS_OK or STREAMOPS_ERR_TIMEOUT and clears it. */
 int streamops_check(streamops_stream_t stream);
+
+/* Number of attempts a wait on an mbarrier inside the bulk-copy pipelines (tuning kind 1) makes
+ * before it gives up; 0 restores the default, 2^22 (seconds). The first attempt is a probe that
+ * never blocks, later ones may each suspend the thread for a hardware-defined time. Exists so that
+ * the give-up path can be exercised: with a limit of 1 a wait gives up at once unless its data is
+ * already there, the kernel sets the error flag, lets the copies it has in flight land (that wait
+ * keeps the full limit) and returns, and streamops_check reports STREAMOPS_ERR_TIMEOUT once. The
+ * output of such a launch is incomplete. Nothing faults and nothing waits without bound. */
+int streamops_set_wait_limit(unsigned tries);
 
 const char *streamops_status_string(int status);
 int streamops_last_cuda_error(void); /* the cudaError_t behind the last STREAMOPS_ERR_CUDA */

@@ -2,8 +2,8 @@
 // Declarations and the contract of every entry point are in include/streamops.h.
 #include <atomic>
 #include <cstring>
+#include <initializer_list>
 #include <mutex>
-#include <vector>
 
 #include "../../include/streamops.h"
 #include "internal.cuh"
@@ -13,27 +13,47 @@ using namespace streamops;
 namespace {
 
 constexpr int kMaxDevices = 64;
+constexpr int kChainRing = 4;           // stages of the host-buffer pipeline: pieces in flight
+
+// One Dot workspace slot of a device. A slot belongs to the stream that used it last: that stream
+// may use it again at once (its Dots run in stream order); another stream may take it over only
+// when the slot's last Dot has finished. Every Dot gets the next sequence number of its slot
+// (`issued`), and the kernel that finishes it writes that number to the slot's word of the device
+// array `done_seq` as its last act: the slot is idle when the two agree. Nothing is added to the
+// stream between kernels (an event record there would end the overlap of dependent launches).
+struct DotSlot {
+    cudaStream_t owner = nullptr;
+    unsigned issued = 0;
+    bool used = false;
+};
 
 struct DeviceState {
-    bool ready = false;
+    std::atomic<bool> ready{false};
     int sm_count = 0;
     double *partials = nullptr;        // kDotSlots * kMaxDotBlocks doubles
     unsigned *tickets = nullptr;       // kDotSlots counters, zero between calls
     int *error_flag = nullptr;         // set by a bounded wait that gave up
-    std::atomic<unsigned> next_slot{0};
+    unsigned *done_seq = nullptr;      // kDotLiveSlots words, see DotSlot
+    unsigned *done_host = nullptr;     // pinned host copy, refreshed only when a slot has to change hands
+    cudaStream_t probe_stream = nullptr;   // carries that refresh, so that no caller's stream is touched
+    std::mutex slot_mutex;
+    DotSlot slots[kDotLiveSlots];      // slots of ordinary calls; the rest serve stream capture
+    unsigned steal_cursor = 0;
+    std::atomic<unsigned> next_capture_slot{0};
     // the array most recently written by an elementwise kernel on this device and the end of it that
     // was written last (1 = high addresses): where its still-cached lines are. Packed into atomics;
     // a stale or torn reading only costs bandwidth.
     std::atomic<uintptr_t> last_written{0};
     std::atomic<size_t> last_written_bytes{0};
     std::atomic<int> last_written_end_high{0};
-    // host-path buffers (streamops_chain_host_*)
-    void *chain_buf[3] = {nullptr, nullptr, nullptr};
+    // host-path ring (streamops_chain_host_*)
+    std::mutex chain_mutex;                            // one host-buffer pass per device at a time
+    void *chain_ring = nullptr;                        // kChainRing stages of three piece buffers each
+    size_t chain_piece_bytes = 0;                      // bytes of one piece buffer in the ring
     void *chain_dot = nullptr;
     double *chain_partials = nullptr;                  // one double per piece
-    size_t chain_bytes = 0;
     cudaStream_t chain_streams[3] = {nullptr, nullptr, nullptr};   // upload, kernels, download
-    std::vector<cudaEvent_t> chain_events;
+    cudaEvent_t chain_uploaded[kChainRing] = {}, chain_computed[kChainRing] = {}, chain_downloaded[kChainRing] = {};
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -71,28 +91,43 @@ streamops_tuning_t default_tuning(int op, int dtype) {
     return t;
 }
 
+// The tuning table. Readers take a copy under the mutex, so a call that runs while another thread
+// changes the table sees either the old or the new entry, never a mixture.
 streamops_tuning_t g_tuning[OP_COUNT][2];
-std::once_flag g_tuning_once;
-void init_tuning() {
+bool g_tuning_ready = false;
+std::mutex g_tuning_mutex;
+void init_tuning_locked() {
     for (int op = 0; op < OP_COUNT; ++op)
         for (int dt = 0; dt < 2; ++dt) g_tuning[op][dt] = default_tuning(op, dt);
+    g_tuning_ready = true;
 }
-const streamops_tuning_t &tuning(int op, int dtype) {
-    std::call_once(g_tuning_once, init_tuning);
+streamops_tuning_t tuning(int op, int dtype) {
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    if (!g_tuning_ready) init_tuning_locked();
     return g_tuning[op][dtype];
 }
+std::atomic<unsigned> g_wait_limit{1u << 22};   // mbarrier.try_wait attempts of the bulk pipelines
 
 int cuda_fail(cudaError_t e) {
     g_last_cuda_error.store((int)e);
     return STREAMOPS_ERR_CUDA;
 }
 
+void free_workspace(DeviceState &d) {
+    cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag); cudaFree(d.done_seq);
+    if (d.done_host) cudaFreeHost(d.done_host);
+    if (d.probe_stream) cudaStreamDestroy(d.probe_stream);
+    d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr; d.done_seq = nullptr;
+    d.done_host = nullptr; d.probe_stream = nullptr;
+    for (DotSlot &s : d.slots) s = DotSlot{};
+}
+
 int init_device(int device, DeviceState **out) {
     if (device < 0 || device >= kMaxDevices) return STREAMOPS_ERR_ARG;
     DeviceState &d = g_dev[device];
-    if (!d.ready) {
+    if (!d.ready.load(std::memory_order_acquire)) {
         std::lock_guard<std::mutex> lock(g_mutex);
-        if (!d.ready) {
+        if (!d.ready.load(std::memory_order_relaxed)) {
             int prev = 0;
             cudaError_t e = cudaGetDevice(&prev);
             if (e != cudaSuccess) return cuda_fail(e);
@@ -103,20 +138,25 @@ int init_device(int device, DeviceState **out) {
                 const size_t pbytes = sizeof(double) * kDotSlots * kMaxDotBlocks;
                 if (cudaMalloc(&d.partials, pbytes) != cudaSuccess ||
                     cudaMalloc(&d.tickets, sizeof(unsigned) * kDotSlots) != cudaSuccess ||
-                    cudaMalloc(&d.error_flag, sizeof(int)) != cudaSuccess) {
+                    cudaMalloc(&d.error_flag, sizeof(int)) != cudaSuccess ||
+                    cudaMalloc(&d.done_seq, sizeof(unsigned) * kDotLiveSlots) != cudaSuccess ||
+                    cudaMallocHost(&d.done_host, sizeof(unsigned) * kDotLiveSlots) != cudaSuccess) {
                     (void)cudaGetLastError();
                     status = STREAMOPS_ERR_WORKSPACE; break;
                 }
                 if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned) * kDotSlots)) != cudaSuccess) { status = cuda_fail(e); break; }
                 if ((e = cudaMemset(d.error_flag, 0, sizeof(int))) != cudaSuccess) { status = cuda_fail(e); break; }
+                if ((e = cudaMemset(d.done_seq, 0, sizeof(unsigned) * kDotLiveSlots)) != cudaSuccess) { status = cuda_fail(e); break; }
+                if ((e = cudaStreamCreateWithFlags(&d.probe_stream, cudaStreamNonBlocking)) != cudaSuccess) { status = cuda_fail(e); break; }
+                for (DotSlot &s : d.slots) s = DotSlot{};
             } while (false);
-            cudaSetDevice(prev);
             if (status != STREAMOPS_OK) {
-                cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag);
-                d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr;
+                free_workspace(d);
+                cudaSetDevice(prev);
                 return status;
             }
-            d.ready = true;
+            cudaSetDevice(prev);
+            d.ready.store(true, std::memory_order_release);
         }
     }
     *out = &d;
@@ -209,6 +249,51 @@ bool valid_tuning(const streamops_tuning_t &t) {
     return true;
 }
 
+// Picks the workspace slot of one Dot call on `stream` and fills in its scratch pointers.
+// Ordinary calls: the slot this stream used last (stream order makes reuse safe), else a slot never
+// used, else a slot whose last Dot has finished (the device's done_seq words are copied to the host
+// on a stream of the library's own: this is the only path that waits for anything, and only for
+// that copy); if all kDotLiveSlots slots are still in flight on other streams, STREAMOPS_ERR_WORKSPACE.
+// Calls made while `stream` is being captured: one of the kDotCaptureSlots slots set aside for graphs,
+// handed out in turn and never shared with ordinary calls; the slot is baked into the graph.
+int acquire_dot_slot(DeviceState *d, cudaStream_t stream, DotScratch *scratch, DotSlot **live) {
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    cudaError_t e = cudaStreamIsCapturing(stream, &capturing);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *live = nullptr;
+    int found = -1;
+    if (capturing != cudaStreamCaptureStatusNone) {
+        found = kDotLiveSlots + (int)(d->next_capture_slot.fetch_add(1) % (unsigned)kDotCaptureSlots);
+        scratch->done = nullptr;
+        scratch->seq = 0;
+    } else {
+        std::lock_guard<std::mutex> lock(d->slot_mutex);
+        for (int i = 0; i < kDotLiveSlots && found < 0; ++i)
+            if (d->slots[i].used && d->slots[i].owner == stream) found = i;
+        for (int i = 0; i < kDotLiveSlots && found < 0; ++i)
+            if (!d->slots[i].used) found = i;
+        if (found < 0) {
+            if ((e = cudaMemcpyAsync(d->done_host, d->done_seq, sizeof(unsigned) * kDotLiveSlots, cudaMemcpyDeviceToHost,
+                                     d->probe_stream)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamSynchronize(d->probe_stream)) != cudaSuccess) return cuda_fail(e);
+            for (int k = 0; k < kDotLiveSlots && found < 0; ++k) {
+                const int i = (int)((d->steal_cursor + (unsigned)k) % (unsigned)kDotLiveSlots);
+                if (d->done_host[i] == d->slots[i].issued) { found = i; d->steal_cursor = (unsigned)i + 1; }
+            }
+        }
+        if (found < 0) return STREAMOPS_ERR_WORKSPACE;
+        DotSlot &s = d->slots[found];
+        s.used = true;
+        s.owner = stream;
+        scratch->done = d->done_seq + found;
+        scratch->seq = ++s.issued;
+        *live = &s;
+    }
+    scratch->partials = d->partials + (size_t)found * kMaxDotBlocks;
+    scratch->ticket = d->tickets + found;
+    return STREAMOPS_OK;
+}
+
 // `wide` (Dot only): out is one double receiving the unrounded total.
 int run_op(int op, int dtype, const void *x, const void *y, void *out, double scalar, size_t n,
            streamops_stream_t stream_, bool wide = false) {
@@ -224,14 +309,11 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
     }
     DeviceState *d = nullptr;
     if ((status = current_device_state(&d)) != STREAMOPS_OK) return status;
-    const streamops_tuning_t &t = tuning(op, dtype);
+    const streamops_tuning_t t = tuning(op, dtype);
 
-    DotScratch scratch{nullptr, nullptr};
-    if (op == OP_DOT) {
-        const unsigned slot = d->next_slot.fetch_add(1) % kDotSlots;
-        scratch.partials = d->partials + (size_t)slot * kMaxDotBlocks;
-        scratch.ticket = d->tickets + slot;
-    }
+    DotScratch scratch{nullptr, nullptr, nullptr, 0};
+    DotSlot *live_slot = nullptr;
+    if (op == OP_DOT && (status = acquire_dot_slot(d, stream, &scratch, &live_slot)) != STREAMOPS_OK) return status;
 
     cudaError_t e;
     int launches = 1;
@@ -243,6 +325,7 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
         b.threads = t.threads;
         b.chunk_bytes = t.chunk_bytes;
         b.stages = t.stages;
+        b.wait_limit = g_wait_limit.load();
         const size_t nchunks = (n * esize + b.chunk_bytes - 1) / b.chunk_bytes;
         size_t grid = (size_t)(t.blocks_per_sm > 0 ? t.blocks_per_sm : 1) * d->sm_count;
         if (grid > nchunks) grid = nchunks;
@@ -272,16 +355,25 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
         } else if (op == OP_DOT) e = launch_dot(dtype, c, t.two_pass != 0, wide, x, y, out, n, scratch, stream, &launches);
         else e = launch_elementwise(op, dtype, c, x, y, out, scalar, n, stream);
     }
-    if (e != cudaSuccess) return cuda_fail(e);
+    if (e != cudaSuccess) {
+        if (live_slot) {                                  // nothing was launched: the slot's count goes back
+            std::lock_guard<std::mutex> lock(d->slot_mutex);
+            --live_slot->issued;
+        }
+        return cuda_fail(e);
+    }
     g_launches.fetch_add((unsigned long long)launches);
     return STREAMOPS_OK;
 }
 
-// Host-buffer pass, pipelined: the arrays are cut into pieces of g_chain_piece_bytes per array; piece k
-// is uploaded on one stream, run through the five kernels on a second (Dot as a double partial sum
-// per piece), and downloaded on a third, so that uploads, kernels and downloads of different pieces
-// overlap and the two directions of the host link are busy at the same time. The dot product is the
-// left-to-right fold of the per-piece partial sums: fixed by n alone, so repeatable bit for bit.
+// Host-buffer pass, pipelined through a small ring of device buffers: the arrays are cut into pieces
+// of g_chain_piece_bytes per array; piece k is uploaded into ring stage k mod kChainRing on one
+// stream, run through the five kernels on a second (Dot as a double partial sum per piece), and
+// downloaded on a third, so that uploads, kernels and downloads of different pieces overlap and the
+// two directions of the host link are busy at the same time. A stage is refilled only after the
+// download of the piece that used it before has finished (an event per stage). Device memory
+// needed: kChainRing x 3 piece buffers, whatever n is. The dot product is the left-to-right fold of
+// the per-piece partial sums: fixed by n and the piece size alone, so repeatable bit for bit.
 std::atomic<size_t> g_chain_piece_bytes{(size_t)16 << 20};
 constexpr size_t kChainMaxPieces = 4096;
 
@@ -292,60 +384,82 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
     DeviceState *d = nullptr;
     int status = current_device_state(&d);
     if (status != STREAMOPS_OK) return status;
-    std::lock_guard<std::mutex> lock(g_mutex);
     cudaError_t e;
-    const size_t bytes = n * sizeof(T);
-    for (cudaStream_t &st : d->chain_streams)
-        if (!st && (e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
-    if (!d->chain_dot && (cudaMalloc(&d->chain_dot, 8) != cudaSuccess ||
-                          cudaMalloc(&d->chain_partials, sizeof(double) * kChainMaxPieces) != cudaSuccess)) {
-        (void)cudaGetLastError();
-        return STREAMOPS_ERR_WORKSPACE;
+    cudaEvent_t end_run = nullptr, end_down = nullptr;
+    {
+        // issuing is serialised per device; the lock is released before the host waits, and a second
+        // caller's work simply queues behind this one's on the same three streams
+        std::lock_guard<std::mutex> lock(d->chain_mutex);
+        for (cudaStream_t &st : d->chain_streams)
+            if (!st && (e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        for (int s = 0; s < kChainRing; ++s)
+            for (cudaEvent_t *ev : {&d->chain_uploaded[s], &d->chain_computed[s], &d->chain_downloaded[s]})
+                if (!*ev && (e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if (!d->chain_dot && (cudaMalloc(&d->chain_dot, 8) != cudaSuccess ||
+                              cudaMalloc(&d->chain_partials, sizeof(double) * kChainMaxPieces) != cudaSuccess)) {
+            (void)cudaGetLastError();
+            return STREAMOPS_ERR_WORKSPACE;
+        }
+        // pieces: whole multiples of 32 bytes, at most kChainMaxPieces of them
+        size_t piece = g_chain_piece_bytes.load() / sizeof(T);
+        while ((n + piece - 1) / piece > kChainMaxPieces) piece *= 2;
+        const size_t pieces = n ? (n + piece - 1) / piece : 0;
+        const size_t piece_bytes = piece * sizeof(T);
+        cudaStream_t up = d->chain_streams[0], run = d->chain_streams[1], down = d->chain_streams[2];
+        if (piece_bytes != d->chain_piece_bytes) {
+            // a ring of another piece size: wait for whatever still uses the old one, then replace it
+            for (cudaStream_t st : d->chain_streams)
+                if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
+            cudaFree(d->chain_ring); d->chain_ring = nullptr; d->chain_piece_bytes = 0;
+            if (cudaMalloc(&d->chain_ring, piece_bytes * 3 * kChainRing) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return STREAMOPS_ERR_WORKSPACE;
+            }
+            d->chain_piece_bytes = piece_bytes;
+        }
+        T *host[3] = {a, b, c};
+        T *dd = (T *)d->chain_dot;
+        for (size_t k = 0; k < pieces; ++k) {
+            const size_t lo = k * piece, len = n - lo < piece ? n - lo : piece;
+            const int s = (int)(k % kChainRing);
+            T *dev[3];
+            for (int i = 0; i < 3; ++i) dev[i] = (T *)((char *)d->chain_ring + ((size_t)s * 3 + i) * piece_bytes);
+            // the stage is free once the download of its previous piece (this call's or an earlier
+            // call's) has finished; an event that was never recorded counts as complete
+            if ((e = cudaStreamWaitEvent(up, d->chain_downloaded[s], 0)) != cudaSuccess) return cuda_fail(e);
+            for (int i = 0; i < 3; ++i)
+                if ((e = cudaMemcpyAsync(dev[i], host[i] + lo, len * sizeof(T), cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventRecord(d->chain_uploaded[s], up)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamWaitEvent(run, d->chain_uploaded[s], 0)) != cudaSuccess) return cuda_fail(e);
+            T *pa = dev[0], *pb = dev[1], *pc = dev[2];
+            // c <- a; b <- s*c; c <- a+b; a <- b+s*c; partial dot(a, b)
+            if ((status = run_op(OP_COPY, dtype, pa, nullptr, pc, scalar, len, run)) != STREAMOPS_OK) return status;
+            if ((status = run_op(OP_SCALE, dtype, pc, nullptr, pb, scalar, len, run)) != STREAMOPS_OK) return status;
+            if ((status = run_op(OP_ADD, dtype, pa, pb, pc, scalar, len, run)) != STREAMOPS_OK) return status;
+            if ((status = run_op(OP_TRIAD, dtype, pb, pc, pa, scalar, len, run)) != STREAMOPS_OK) return status;
+            if ((status = run_op(OP_DOT, dtype, pa, pb, d->chain_partials + k, scalar, len, run, dtype == DT_F32)) != STREAMOPS_OK) return status;
+            if ((e = cudaEventRecord(d->chain_computed[s], run)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamWaitEvent(down, d->chain_computed[s], 0)) != cudaSuccess) return cuda_fail(e);
+            for (int i = 0; i < 3; ++i)
+                if ((e = cudaMemcpyAsync(host[i] + lo, dev[i], len * sizeof(T), cudaMemcpyDeviceToHost, down)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventRecord(d->chain_downloaded[s], down)) != cudaSuccess) return cuda_fail(e);
+        }
+        if ((e = launch_fold(dtype, d->chain_partials, pieces, dd, run)) != cudaSuccess) return cuda_fail(e);
+        g_launches.fetch_add(1);
+        if ((e = cudaMemcpyAsync(dot_out, dd, sizeof(T), cudaMemcpyDeviceToHost, run)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&end_run, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&end_down, cudaEventDisableTiming)) != cudaSuccess) { cudaEventDestroy(end_run); return cuda_fail(e); }
+        e = cudaEventRecord(end_run, run);
+        if (e == cudaSuccess) e = cudaEventRecord(end_down, down);
+        if (e != cudaSuccess) { cudaEventDestroy(end_run); cudaEventDestroy(end_down); return cuda_fail(e); }
     }
-    if (bytes > d->chain_bytes) {
-        for (void *&p : d->chain_buf) { cudaFree(p); p = nullptr; }
-        d->chain_bytes = 0;
-        for (void *&p : d->chain_buf)
-            if (cudaMalloc(&p, bytes) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_ERR_WORKSPACE; }
-        d->chain_bytes = bytes;
-    }
-    // pieces: whole multiples of 32 bytes, at most kChainMaxPieces of them
-    size_t piece = g_chain_piece_bytes.load() / sizeof(T);
-    while ((n + piece - 1) / piece > kChainMaxPieces) piece *= 2;
-    const size_t pieces = n ? (n + piece - 1) / piece : 0;
-    while (d->chain_events.size() < 2 * pieces) {
-        cudaEvent_t ev;
-        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-        d->chain_events.push_back(ev);
-    }
-    cudaStream_t up = d->chain_streams[0], run = d->chain_streams[1], down = d->chain_streams[2];
-    T *host[3] = {a, b, c};
-    T *dev[3] = {(T *)d->chain_buf[0], (T *)d->chain_buf[1], (T *)d->chain_buf[2]};
-    T *dd = (T *)d->chain_dot;
-    for (size_t k = 0; k < pieces; ++k) {
-        const size_t lo = k * piece, len = n - lo < piece ? n - lo : piece;
-        cudaEvent_t uploaded = d->chain_events[2 * k], computed = d->chain_events[2 * k + 1];
-        for (int i = 0; i < 3; ++i)
-            if ((e = cudaMemcpyAsync(dev[i] + lo, host[i] + lo, len * sizeof(T), cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaEventRecord(uploaded, up)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaStreamWaitEvent(run, uploaded, 0)) != cudaSuccess) return cuda_fail(e);
-        T *pa = dev[0] + lo, *pb = dev[1] + lo, *pc = dev[2] + lo;
-        // c <- a; b <- s*c; c <- a+b; a <- b+s*c; partial dot(a, b)
-        if ((status = run_op(OP_COPY, dtype, pa, nullptr, pc, scalar, len, run)) != STREAMOPS_OK) return status;
-        if ((status = run_op(OP_SCALE, dtype, pc, nullptr, pb, scalar, len, run)) != STREAMOPS_OK) return status;
-        if ((status = run_op(OP_ADD, dtype, pa, pb, pc, scalar, len, run)) != STREAMOPS_OK) return status;
-        if ((status = run_op(OP_TRIAD, dtype, pb, pc, pa, scalar, len, run)) != STREAMOPS_OK) return status;
-        if ((status = run_op(OP_DOT, dtype, pa, pb, d->chain_partials + k, scalar, len, run, dtype == DT_F32)) != STREAMOPS_OK) return status;
-        if ((e = cudaEventRecord(computed, run)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaStreamWaitEvent(down, computed, 0)) != cudaSuccess) return cuda_fail(e);
-        for (int i = 0; i < 3; ++i)
-            if ((e = cudaMemcpyAsync(host[i] + lo, dev[i] + lo, len * sizeof(T), cudaMemcpyDeviceToHost, down)) != cudaSuccess) return cuda_fail(e);
-    }
-    if ((e = launch_fold(dtype, d->chain_partials, pieces, dd, run)) != cudaSuccess) return cuda_fail(e);
-    g_launches.fetch_add(1);
-    if ((e = cudaMemcpyAsync(dot_out, dd, sizeof(T), cudaMemcpyDeviceToHost, run)) != cudaSuccess) return cuda_fail(e);
-    for (cudaStream_t st : d->chain_streams)
-        if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
+    // this call's own work only: the kernels and the dot product, then the last download
+    e = cudaEventSynchronize(end_run);
+    const cudaError_t e2 = cudaEventSynchronize(end_down);
+    cudaEventDestroy(end_run);
+    cudaEventDestroy(end_down);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (e2 != cudaSuccess) return cuda_fail(e2);
     return STREAMOPS_OK;
 }
 
@@ -443,17 +557,22 @@ int streamops_shutdown(void) {
     if (cudaGetDevice(&prev) != cudaSuccess) { (void)cudaGetLastError(); return STREAMOPS_OK; }
     for (int i = 0; i < kMaxDevices; ++i) {
         DeviceState &d = g_dev[i];
-        if (!d.ready) continue;
+        if (!d.ready.load(std::memory_order_acquire)) continue;
         cudaSetDevice(i);
         cudaDeviceSynchronize();
-        cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag); cudaFree(d.chain_dot);
-        for (void *&p : d.chain_buf) { cudaFree(p); p = nullptr; }
+        free_workspace(d);
+        cudaFree(d.chain_dot);
+        cudaFree(d.chain_ring); d.chain_ring = nullptr; d.chain_piece_bytes = 0;
         cudaFree(d.chain_partials); d.chain_partials = nullptr;
         for (cudaStream_t &st : d.chain_streams) { if (st) cudaStreamDestroy(st); st = nullptr; }
-        for (cudaEvent_t ev : d.chain_events) cudaEventDestroy(ev);
-        d.chain_events.clear();
-        d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr; d.chain_dot = nullptr;
-        d.chain_bytes = 0; d.ready = false;
+        for (int s = 0; s < kChainRing; ++s)
+            for (cudaEvent_t *ev : {&d.chain_uploaded[s], &d.chain_computed[s], &d.chain_downloaded[s]}) {
+                if (*ev) cudaEventDestroy(*ev);
+                *ev = nullptr;
+            }
+        d.chain_dot = nullptr;
+        d.last_written.store(0);
+        d.ready.store(false, std::memory_order_release);
     }
     cudaSetDevice(prev);
     return STREAMOPS_OK;
@@ -462,7 +581,8 @@ int streamops_shutdown(void) {
 int streamops_set_tuning(int op, int dtype, const streamops_tuning_t *t) {
     if (!t) return STREAMOPS_ERR_NULL;
     if (op < 0 || op >= OP_COUNT || dtype < 0 || dtype > 1 || !valid_tuning(*t)) return STREAMOPS_ERR_ARG;
-    (void)tuning(op, dtype);
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    if (!g_tuning_ready) init_tuning_locked();
     g_tuning[op][dtype] = *t;
     return STREAMOPS_OK;
 }
@@ -475,8 +595,8 @@ int streamops_get_tuning(int op, int dtype, streamops_tuning_t *t) {
 }
 
 int streamops_reset_tuning(void) {
-    (void)tuning(0, 0);
-    init_tuning();
+    std::lock_guard<std::mutex> lock(g_tuning_mutex);
+    init_tuning_locked();
     return STREAMOPS_OK;
 }
 
@@ -515,12 +635,17 @@ const char *streamops_status_string(int status) {
         case STREAMOPS_ERR_ALIGN: return "pointer not aligned to the element size";
         case STREAMOPS_ERR_OVERLAP: return "output partially overlaps an input";
         case STREAMOPS_ERR_CUDA: return "CUDA error (see streamops_last_cuda_error)";
-        case STREAMOPS_ERR_WORKSPACE: return "workspace allocation failed";
+        case STREAMOPS_ERR_WORKSPACE: return "workspace unavailable (allocation failed, or every Dot slot is in flight)";
         case STREAMOPS_ERR_TIMEOUT: return "a bounded wait inside a kernel gave up";
         case STREAMOPS_ERR_ARG: return "argument out of range";
         case STREAMOPS_ERR_TOO_LARGE: return "n exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
+}
+
+int streamops_set_wait_limit(unsigned tries) {
+    g_wait_limit.store(tries == 0 ? (1u << 22) : tries);
+    return STREAMOPS_OK;
 }
 
 int streamops_last_cuda_error(void) { return g_last_cuda_error.load(); }

@@ -18,9 +18,11 @@
 //                            into per-thread double accumulators, then the shared fixed-order
 //                            reduction).
 //
-// Every wait on an mbarrier is a bounded loop around mbarrier.try_wait. A wait that runs out
-// writes a code to the device error flag, tells the rest of the CTA to stop, waits (bounded) for
-// the copies already in flight, and returns; the host reports STREAMOPS_ERR_TIMEOUT.
+// Every wait on an mbarrier is a bounded loop around mbarrier.try_wait (`wait_limit` attempts, a
+// kernel argument: 2^22 by default, lowered by streamops_set_wait_limit to exercise this path). A
+// wait that runs out writes a code to the device error flag and tells the rest of the CTA to stop;
+// the loading thread always waits (bounded) for the copies it has in flight before it returns;
+// the host reports STREAMOPS_ERR_TIMEOUT. The output of such a launch is incomplete.
 #include "internal.cuh"
 #include "memops.cuh"
 #include "reduce.cuh"
@@ -29,7 +31,7 @@ namespace streamops {
 
 namespace {
 
-constexpr unsigned kWaitLimit = 1u << 22;   // try_wait attempts before giving up
+constexpr unsigned kDrainLimit = 1u << 22;  // try_wait attempts granted to copies already in flight
 constexpr int kMaxStages = 8;
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) {
@@ -56,9 +58,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity) {
                  : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait; false = gave up (or another thread of the CTA already did).
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity, volatile int *stop) {
-    for (unsigned i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait of at most `limit` attempts; false = gave up (or another thread of the CTA already did).
+// The first attempt is a probe that never blocks (test_wait); each later one (try_wait) may suspend
+// the thread for a hardware-defined time before it reports "not yet". A limit of 1 therefore gives up
+// at once unless the phase has already completed.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity, volatile int *stop, unsigned limit) {
+    if (mbar_test_wait(bar, parity)) return true;
+    for (unsigned i = 1; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 1023u) == 1023u && *stop) return false;
     }
@@ -107,13 +121,16 @@ struct Ring {
     int stop;
 };
 
-// After a failed wait: give the copies already issued a bounded chance to land, so that no
-// copy is still writing into this CTA's shared memory when it exits.
+// Last act of every loading thread, whether its loop ended normally or a wait gave up: wait
+// (bounded, with the full fixed limit whatever limit the pipeline's own waits run under) until
+// the copies it issued last have landed, so that no copy is still writing into this CTA's shared
+// memory when the CTA exits. Each of those copies was armed on its stage's "full" barrier, and a
+// completed phase stays completed, so this returns at once when the data is already there.
 __device__ __forceinline__ void drain_loads(Ring *ring, int stages, size_t issued) {
     int dummy = 0;
     const size_t first = issued > (size_t)stages ? issued - stages : 0;
     for (size_t it = first; it < issued; ++it)
-        mbar_wait(&ring->full[it % stages], (unsigned)((it / stages) & 1), &dummy);
+        mbar_wait(&ring->full[it % stages], (unsigned)((it / stages) & 1), &dummy, kDrainLimit);
 }
 
 __device__ __forceinline__ void flag_timeout(Ring *ring, int *error_flag, int code) {
@@ -124,7 +141,8 @@ __device__ __forceinline__ void flag_timeout(Ring *ring, int *error_flag, int co
 // ------------------------------------------------------------------------------------ Copy
 // 64 threads: warp 0 lane 0 loads, warp 1 lane 0 stores; the other lanes only move the tail.
 __global__ void __launch_bounds__(64)
-bulk_copy_kernel(const char *x, char *out, size_t total_bytes, unsigned chunk, int stages, int *error_flag) {
+bulk_copy_kernel(const char *x, char *out, size_t total_bytes, unsigned chunk, int stages, int *error_flag,
+                 unsigned wait_limit) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ Ring ring;
     const Chunks ck = make_chunks(total_bytes, chunk);
@@ -140,19 +158,19 @@ bulk_copy_kernel(const char *x, char *out, size_t total_bytes, unsigned chunk, i
         for (size_t k = blockIdx.x; k < ck.nchunks; k += gridDim.x, ++it) {
             const int s = (int)(it % stages);
             const unsigned ph = (unsigned)((it / stages) & 1);
-            if (!mbar_wait(&ring.empty[s], ph ^ 1u, &ring.stop)) { flag_timeout(&ring, error_flag, 1); break; }
+            if (!mbar_wait(&ring.empty[s], ph ^ 1u, &ring.stop, wait_limit)) { flag_timeout(&ring, error_flag, 1); break; }
             const unsigned bytes = ck.size_of(k);
             mbar_arrive_expect_tx(&ring.full[s], bytes);
             bulk_load(smem + (size_t)s * chunk, x + k * (size_t)chunk, bytes, &ring.full[s]);
         }
-        if (ring.stop) drain_loads(&ring, stages, it);
+        drain_loads(&ring, stages, it);
     } else if (threadIdx.x == 32) {                           // storer
         size_t it = 0;
         bool ok = true;
         for (size_t k = blockIdx.x; k < ck.nchunks; k += gridDim.x, ++it) {
             const int s = (int)(it % stages);
             const unsigned ph = (unsigned)((it / stages) & 1);
-            if (!mbar_wait(&ring.full[s], ph, &ring.stop)) { flag_timeout(&ring, error_flag, 2); ok = false; break; }
+            if (!mbar_wait(&ring.full[s], ph, &ring.stop, wait_limit)) { flag_timeout(&ring, error_flag, 2); ok = false; break; }
             bulk_store(out + k * (size_t)chunk, smem + (size_t)s * chunk, ck.size_of(k));
             bulk_commit();
             if (it > 0) {                                     // the previous store has left its stage
@@ -191,7 +209,8 @@ __device__ __forceinline__ T apply(T x, T y, T s) {
 template <typename T, int OP, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads + 32)
 bulk_compute_kernel(const T *x, const T *y, T *out, T s, size_t n, unsigned chunk, int stages,
-                    double *partials, unsigned *ticket, int *error_flag) {
+                    double *partials, unsigned *ticket, int *error_flag, unsigned wait_limit,
+                    unsigned *done, unsigned seq) {
     constexpr bool USES_Y = (OP != OP_SCALE);
     constexpr int EPV = 16 / (int)sizeof(T);
     extern __shared__ __align__(128) unsigned char smem[];
@@ -220,21 +239,21 @@ bulk_compute_kernel(const T *x, const T *y, T *out, T s, size_t n, unsigned chun
             for (size_t k = blockIdx.x; k < ck.nchunks; k += gridDim.x, ++it) {
                 const int st = (int)(it % stages);
                 const unsigned ph = (unsigned)((it / stages) & 1);
-                if (!mbar_wait(&ring.empty[st], ph ^ 1u, &ring.stop)) { flag_timeout(&ring, error_flag, 3); break; }
+                if (!mbar_wait(&ring.empty[st], ph ^ 1u, &ring.stop, wait_limit)) { flag_timeout(&ring, error_flag, 3); break; }
                 const unsigned bytes = ck.size_of(k);
                 unsigned char *stage = smem + (size_t)st * stage_bytes;
                 mbar_arrive_expect_tx(&ring.full[st], USES_Y ? 2 * bytes : bytes);
                 bulk_load(stage, xb + k * (size_t)chunk, bytes, &ring.full[st]);
                 if constexpr (USES_Y) bulk_load(stage + chunk, yb + k * (size_t)chunk, bytes, &ring.full[st]);
             }
-            if (ring.stop) drain_loads(&ring, stages, it);
+            drain_loads(&ring, stages, it);
         }
     } else {
         size_t it = 0;
         for (size_t k = blockIdx.x; k < ck.nchunks; k += gridDim.x, ++it) {
             const int st = (int)(it % stages);
             const unsigned ph = (unsigned)((it / stages) & 1);
-            if (!mbar_wait(&ring.full[st], ph, &ring.stop)) { flag_timeout(&ring, error_flag, 4); break; }
+            if (!mbar_wait(&ring.full[st], ph, &ring.stop, wait_limit)) { flag_timeout(&ring, error_flag, 4); break; }
             const unsigned bytes = ck.size_of(k);
             const unsigned char *stage = smem + (size_t)st * stage_bytes;
             char *dst = ob + k * (size_t)chunk;
@@ -267,7 +286,7 @@ bulk_compute_kernel(const T *x, const T *y, T *out, T s, size_t n, unsigned chun
     }
     if constexpr (OP == OP_DOT) {
         const double bsum = block_sum(acc, warp_part);
-        publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last);
+        publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, done, seq);
     }
 }
 
@@ -284,7 +303,7 @@ cudaError_t launch_compute(const BulkLaunch &c, const T *x, const T *y, T *out, 
     cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return e;
     kernel<<<c.grid, c.threads + 32, smem, st>>>(x, y, out, (T)scalar, n, (unsigned)c.chunk_bytes, c.stages,
-                                                 sc.partials, sc.ticket, error_flag);
+                                                 sc.partials, sc.ticket, error_flag, c.wait_limit, sc.done, sc.seq);
     return cudaGetLastError();
 }
 
@@ -321,7 +340,7 @@ cudaError_t launch_bulk(int op, int dtype, const BulkLaunch &c, const void *x, c
         if (e != cudaSuccess) return e;
         const size_t bytes = n * (dtype == DT_F64 ? 8 : 4);
         bulk_copy_kernel<<<c.grid, 64, smem, stream>>>((const char *)x, (char *)out, bytes,
-                                                       (unsigned)c.chunk_bytes, c.stages, error_flag);
+                                                       (unsigned)c.chunk_bytes, c.stages, error_flag, c.wait_limit);
         return cudaGetLastError();
     }
     if (dtype == DT_F64)

@@ -30,7 +30,8 @@ __device__ __forceinline__ double fold_vec(double acc, const Vec<VB> &xv, const 
 
 template <typename T, int VB, int U, int POL, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads)
-dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int reverse) {
+dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int reverse,
+                 unsigned *done, unsigned seq) {
     constexpr int EPV = VB / (int)sizeof(T);
     __shared__ double warp_part[32];
     __shared__ bool is_last;
@@ -71,20 +72,22 @@ dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *t
     for (int u = 1; u < U; ++u) tsum += acc[u];
     const double bsum = block_sum(tsum, warp_part);
 
-    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last);
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, done, seq);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(1024)
-dot_pass2_kernel(const double *partials, unsigned count, T *out) {
+dot_pass2_kernel(const double *partials, unsigned count, T *out, unsigned *done, unsigned seq) {
     __shared__ double warp_part[32];
     finish<T>(partials, count, out, warp_part);
+    if (threadIdx.x == 0) mark_done(done, seq);
 }
 
 // Scalar pass 1 for pointers that are not 16-byte aligned: same structure, one element per load.
 template <typename T, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads)
-dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out) {
+dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out,
+                  unsigned *done, unsigned seq) {
     __shared__ double warp_part[32];
     __shared__ bool is_last;
     double acc = 0.0;
@@ -92,13 +95,13 @@ dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
         acc = fma(widen<T>(x[i]), widen<T>(y[i]), acc);
     const double bsum = block_sum(acc, warp_part);
-    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last);
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, done, seq);
 }
 
 template <typename T, int VB, int U, bool SL>
 cudaError_t launch_pol(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
     switch (c.policy) {
-#define STREAMOPS_CASE(P) case P: return launch_kernel(dot_pass1_kernel<T, VB, U, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, c.reverse);
+#define STREAMOPS_CASE(P) case P: return launch_kernel(dot_pass1_kernel<T, VB, U, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, c.reverse, s.done, s.seq);
         STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4) STREAMOPS_CASE(5) STREAMOPS_CASE(6)
 #undef STREAMOPS_CASE
         default: return cudaErrorInvalidValue;
@@ -120,7 +123,7 @@ template <typename T, bool SL>
 cudaError_t launch_pass1(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
     if (c.vec_bytes == 32) return launch_unroll<T, 32, SL>(c, x, y, n, s, out, st);
     if (c.vec_bytes == 16) return launch_unroll<T, 16, SL>(c, x, y, n, s, out, st);
-    dot_scalar_kernel<T, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out);
+    dot_scalar_kernel<T, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out, s.done, s.seq);
     return cudaGetLastError();
 }
 
@@ -140,7 +143,7 @@ cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, bool wide, const T *
         *launches = 2;
         cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, (T *)nullptr, st);
         if (e != cudaSuccess) return e;
-        dot_pass2_kernel<double><<<1, 1024, 0, st>>>(s.partials, c.grid, (double *)out);
+        dot_pass2_kernel<double><<<1, 1024, 0, st>>>(s.partials, c.grid, (double *)out, s.done, s.seq);
         return cudaGetLastError();
     }
     T *o = (T *)out;
@@ -151,7 +154,7 @@ cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, bool wide, const T *
     *launches = 2;
     cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, o, st);
     if (e != cudaSuccess) return e;
-    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, o);
+    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, o, s.done, s.seq);
     return cudaGetLastError();
 }
 

@@ -73,7 +73,8 @@ __device__ __forceinline__ Pair block_merge(Pair v, Pair *warp_part) {
 
 template <typename T, int U>
 __global__ void __launch_bounds__(kMaxThreads, 2)
-dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int vectorised) {
+dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int vectorised,
+                unsigned *done, unsigned seq) {
     constexpr int EPV = 32 / (int)sizeof(T);
     __shared__ Pair warp_part[32];
     __shared__ bool is_last;
@@ -134,6 +135,7 @@ dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ti
         if (threadIdx.x == 0) {
             out[0] = (T)__dadd_rn(total.s, total.c);
             *ticket = 0u;
+            mark_done(done, seq);
         }
     }
 }
@@ -142,9 +144,9 @@ template <typename T>
 cudaError_t launch_t(const VecLaunch &c, const T *x, const T *y, T *out, size_t n, const DotScratch &s, cudaStream_t st) {
     const int vec = c.vec_bytes == 32;
     switch (vec ? c.unroll : 1) {
-        case 1: return launch_kernel(dot_comp_kernel<T, 1>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec);
-        case 2: return launch_kernel(dot_comp_kernel<T, 2>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec);
-        case 4: return launch_kernel(dot_comp_kernel<T, 4>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec);
+        case 1: return launch_kernel(dot_comp_kernel<T, 1>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.done, s.seq);
+        case 2: return launch_kernel(dot_comp_kernel<T, 2>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.done, s.seq);
+        case 4: return launch_kernel(dot_comp_kernel<T, 4>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.done, s.seq);
         default: return cudaErrorInvalidValue;
     }
 }

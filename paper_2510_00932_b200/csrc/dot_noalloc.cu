@@ -16,6 +16,7 @@
 #include <mutex>
 
 #include "../../include/streamops.h"
+#include "internal.cuh"
 #include "memops.cuh"
 #include "reduce.cuh"
 
@@ -78,7 +79,7 @@ dot_noalloc_kernel(const double *x, const double *y, size_t n, double *scratch, 
     }
     const double tsum = ((acc[0] + acc[1]) + acc[2]) + acc[3];
     const double bsum = block_sum(tsum, warp_part);
-    publish_partial<double, true>(bsum, partials, ticket, out, warp_part, &is_last);
+    publish_partial<double, true>(bsum, partials, ticket, out, warp_part, &is_last, nullptr, 0u);
 }
 
 // Device address of the scratch array, looked up once per device with that device current.
@@ -117,15 +118,18 @@ extern "C" int stream_dot_noalloc_f64(const double *x, const double *y, double *
     if (((uintptr_t)out % 8) || (n > 0 && (((uintptr_t)x % 8) || ((uintptr_t)y % 8)))) return STREAMOPS_ERR_ALIGN;
     if (n > (size_t)STREAMOPS_DOT_NOALLOC_MAX_N) return STREAMOPS_ERR_TOO_LARGE;
     if (n > 0 && (overlaps(x, n * 8, out, 8) || overlaps(y, n * 8, out, 8))) return STREAMOPS_ERR_OVERLAP;
-    if (n == 0) return cudaMemsetAsync(out, 0, sizeof(double), stream) == cudaSuccess ? STREAMOPS_OK : STREAMOPS_ERR_CUDA;
+    cudaError_t e;
+    if (n == 0) return (e = cudaMemsetAsync(out, 0, sizeof(double), stream)) == cudaSuccess ? STREAMOPS_OK : note_cuda_error(e);
 
     double *scratch = nullptr;
-    if (scratch_for_current_device(&scratch) != cudaSuccess) return STREAMOPS_ERR_CUDA;
+    if ((e = scratch_for_current_device(&scratch)) != cudaSuccess) return note_cuda_error(e);
     // the array keeps the last call's contents: the ticket must start at zero (an interrupted
     // earlier call could have left it mid-count); the partial sums are all rewritten before use
-    if (cudaMemsetAsync(scratch + kTicketSlot, 0, sizeof(unsigned), stream) != cudaSuccess) return STREAMOPS_ERR_CUDA;
+    if ((e = cudaMemsetAsync(scratch + kTicketSlot, 0, sizeof(unsigned), stream)) != cudaSuccess) return note_cuda_error(e);
     const unsigned blocks = (unsigned)((n + kSpan - 1) / kSpan);
     const int vectorised = (((uintptr_t)x | (uintptr_t)y) & 31) == 0;
     dot_noalloc_kernel<<<blocks, kThreads, 0, stream>>>(x, y, n, scratch, out, vectorised);
-    return cudaGetLastError() == cudaSuccess ? STREAMOPS_OK : STREAMOPS_ERR_CUDA;
+    if ((e = cudaGetLastError()) != cudaSuccess) return note_cuda_error(e);
+    note_launches(1);                      // host-side counters: nothing here allocates
+    return STREAMOPS_OK;
 }

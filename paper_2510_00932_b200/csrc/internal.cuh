@@ -11,7 +11,9 @@ enum : int { DT_F32 = 0, DT_F64 = 1 };
 
 constexpr int kMaxThreads = 512;       // __launch_bounds__ of every vector kernel
 constexpr int kMaxDotBlocks = 16384;   // partial sums per Dot workspace slot
-constexpr int kDotSlots = 32;          // Dot calls that may be in flight per device
+constexpr int kDotLiveSlots = 24;      // Dot calls on different streams that may be in flight per device
+constexpr int kDotCaptureSlots = 8;    // slots set aside for Dot calls recorded into CUDA graphs
+constexpr int kDotSlots = kDotLiveSlots + kDotCaptureSlots;
 
 // Resolved launch shape for the register-vector kernels.
 struct VecLaunch {
@@ -32,6 +34,7 @@ struct BulkLaunch {
     unsigned grid;
     int chunk_bytes;
     int stages;
+    unsigned wait_limit;   // mbarrier.try_wait attempts before a pipeline wait gives up
 };
 
 // Launch helper. With `pdl` the kernel is launched with programmatic stream serialization: its
@@ -68,6 +71,8 @@ __device__ __forceinline__ void grid_dependency_sync() {
 struct DotScratch {
     double *partials;      // kMaxDotBlocks doubles
     unsigned *ticket;      // one counter, zero between calls
+    unsigned *done;        // where the kernel that finishes the Dot writes `seq` as its last act (may be null)
+    unsigned seq;          // this call's sequence number on its slot
 };
 
 // api.cu: bookkeeping shared by the entry points that live in other files

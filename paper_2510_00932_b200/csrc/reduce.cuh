@@ -38,11 +38,21 @@ __device__ __forceinline__ void finish(const double *partials, unsigned count, T
     if (threadIdx.x == 0) out[0] = (T)total;
 }
 
+// Last act of the thread that finishes a Dot: after everything it read or wrote in the slot's
+// scratch, it publishes the call's sequence number, which tells the host (when it needs to know)
+// that the slot is free for another stream.
+__device__ __forceinline__ void mark_done(unsigned *done, unsigned seq) {
+    if (done) {
+        __threadfence();
+        *done = seq;
+    }
+}
+
 // Publishes this block's partial sum; in the single-launch form the block that arrives last at
 // the ticket then folds all partials (in block-index order) and re-arms the ticket.
 template <typename T, bool SINGLE_LAUNCH>
 __device__ __forceinline__ void publish_partial(double bsum, double *partials, unsigned *ticket, T *out,
-                                                double *warp_part, bool *is_last) {
+                                                double *warp_part, bool *is_last, unsigned *done, unsigned seq) {
     if (threadIdx.x == 0) partials[blockIdx.x] = bsum;
     if constexpr (SINGLE_LAUNCH) {
         if (threadIdx.x == 0) {
@@ -54,7 +64,10 @@ __device__ __forceinline__ void publish_partial(double bsum, double *partials, u
         if (*is_last) {
             __threadfence();
             finish<T>(partials, gridDim.x, out, warp_part);
-            if (threadIdx.x == 0) *ticket = 0u;               // ready for the next call
+            if (threadIdx.x == 0) {
+                *ticket = 0u;                                 // ready for the next call
+                mark_done(done, seq);
+            }
         }
     }
 }

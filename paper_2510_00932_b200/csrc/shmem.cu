@@ -18,6 +18,8 @@
 // No thread ever reads a column another thread writes, so there is no barrier in the loop --
 // the time is shared-memory bandwidth: 2 * rounds * 4 bytes per word, against 128 bytes per
 // clock per SM.
+#include <atomic>
+
 #include "../../include/streamops.h"
 #include "internal.cuh"
 
@@ -120,7 +122,7 @@ shmem_mix_kernel(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n) {
     }
 }
 
-int g_width_bytes = 16;
+std::atomic<int> g_width_bytes{16};
 
 template <int VW>
 cudaError_t launch_width(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n, int sm_count, cudaStream_t st) {
@@ -154,7 +156,7 @@ extern "C" int shmem_mix_u32(const unsigned *x, unsigned *out, unsigned rounds, 
     cudaError_t e = cudaGetDevice(&device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e != cudaSuccess) return note_cuda_error(e);
-    int width = g_width_bytes;
+    int width = g_width_bytes.load();
     const uintptr_t bits = x0 | o0;
     while (width > 4 && (bits % (uintptr_t)width)) width >>= 1;          // narrower pieces for less aligned arrays
     if (width == 16) e = launch_width<4>(x, out, rounds, n, sm_count, stream);
@@ -167,8 +169,8 @@ extern "C" int shmem_mix_u32(const unsigned *x, unsigned *out, unsigned rounds, 
 
 extern "C" int streamops_set_shmem_width(int bytes) {
     if (bytes != 4 && bytes != 8 && bytes != 16) return STREAMOPS_ERR_ARG;
-    g_width_bytes = bytes;
+    g_width_bytes.store(bytes);
     return STREAMOPS_OK;
 }
 
-extern "C" int streamops_get_shmem_width(void) { return g_width_bytes; }
+extern "C" int streamops_get_shmem_width(void) { return g_width_bytes.load(); }

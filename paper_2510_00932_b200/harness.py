@@ -151,3 +151,49 @@ def per_op_report(durations_ms: dict, n: int, itemsize: int, peak_gbs: float) ->
         out[op] = {"ms": round(ms, 5), "gbs": round(gbs, 1), "frac_measured_peak": round(gbs / peak_gbs, 4),
                    "frac_nominal_8tbs": round(gbs / NOMINAL_HBM_GBS, 4)}
     return out
+
+
+def launch_ranks(script: str, argv: list, nproc: int, extra_env: dict | None = None) -> int:
+    """Starts `nproc` ranks of `script argv...` on this node with torch.distributed.run (one process
+    per GPU, rendezvous on 127.0.0.1 at a free port) and returns the launcher's exit code. NCCL's
+    initialisation log is switched on (to stderr) unless the caller configured NCCL_DEBUG, so that
+    the communicator's size can be read off a run's output."""
+    import socket
+    import sys
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    if "NCCL_DEBUG" not in env:
+        env.update(NCCL_DEBUG="INFO", NCCL_DEBUG_SUBSYS="INIT", NCCL_DEBUG_FILE="/dev/stderr")
+    env.update(extra_env or {})
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(nproc)}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), script, *argv]
+    return subprocess.call(cmd, env=env)
+
+
+def traffic_file(workload: str) -> str:
+    return os.path.join(ROOT, "profiles", f"ncu_dram_traffic_opmajor_{workload}.txt")
+
+
+def read_traffic_file(path: str):
+    """The JSON object stored after the '#' comment lines of a traffic summary, or None."""
+    try:
+        with open(path) as f:
+            body = "".join(line for line in f if not line.lstrip().startswith("#"))
+        return json.loads(body)
+    except (OSError, ValueError):
+        return None
+
+
+def captured_traffic(workload: str, op: str, tuning: dict):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of `op` from the stored
+    ncu capture of this workload, or None when there is no capture or when it was taken under a
+    tuning other than the one in force (the kernel has changed since)."""
+    data = read_traffic_file(traffic_file(workload))
+    if not data:
+        return None
+    entry = data.get("kernels", {}).get(op)
+    if not entry or entry.get("tuning") != tuning:
+        return None
+    return int(entry["dram_read_bytes"] + entry["dram_write_bytes"])

@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.streamops_reset_tuning.argtypes, L.streamops_reset_tuning.restype = [], ci
         L.streamops_policy_name.argtypes, L.streamops_policy_name.restype = [ci], ctypes.c_char_p
         L.streamops_check.argtypes, L.streamops_check.restype = [vp], ci
+        L.streamops_set_wait_limit.argtypes, L.streamops_set_wait_limit.restype = [ctypes.c_uint], ci
         L.streamops_status_string.argtypes, L.streamops_status_string.restype = [ci], ctypes.c_char_p
         L.streamops_last_cuda_error.argtypes, L.streamops_last_cuda_error.restype = [], ci
         L.streamops_launch_count.argtypes, L.streamops_launch_count.restype = [], ctypes.c_ulonglong
@@ -97,6 +98,7 @@ def _raise(status: int):
 
 _SUFFIX = None            # torch dtype -> "f32" / "f64", filled on first use
 _raw_stream = None        # fast accessor of the current stream's handle
+_current_device = None    # fast accessor of the current CUDA device index
 
 
 def _suffix(t) -> str:
@@ -113,7 +115,7 @@ def _suffix(t) -> str:
 def _marshal(*tensors):
     """Common dtype suffix and the current stream handle of the tensors' device. Kept lean: at
     L2-resident sizes a kernel lasts a few microseconds and this code is what the host spends."""
-    global _raw_stream
+    global _raw_stream, _current_device
     first = tensors[0]
     suf = _suffix(first)
     dev = first.get_device()
@@ -128,6 +130,11 @@ def _marshal(*tensors):
         import torch
         _raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None) or (
             lambda d: torch.cuda.current_stream(d).cuda_stream)
+        _current_device = getattr(torch._C, "_cuda_getDevice", None) or torch.cuda.current_device
+    # the library takes its per-device state (Dot workspace, SM count) from the CURRENT device
+    if dev != _current_device():
+        raise ValueError(f"tensors live on cuda:{dev} but the current device is cuda:{_current_device()}; "
+                         "make the tensors' device current (torch.cuda.device) around the call")
     return suf, _raw_stream(dev)
 
 
@@ -181,6 +188,8 @@ def dot_wide(x, y, out64):
     out64 is a one-element float64 device tensor (stream_dot_wide_f32 / stream_dot_f64)."""
     import torch
     suf, stream = _marshal(x, y)
+    if out64.is_cuda and out64.get_device() != x.get_device():
+        raise ValueError("all tensors of one call share a device")
     if x.numel() != y.numel() or out64.numel() != 1 or out64.dtype != torch.float64 or not out64.is_cuda:
         raise ValueError("dot_wide takes two equal-length inputs and a one-element float64 device output")
     f = lib().stream_dot_f64 if suf == "f64" else lib().stream_dot_wide_f32
@@ -194,8 +203,8 @@ def fold(partials, out):
     if partials.dtype != torch.float64 or not partials.is_cuda or not partials.is_contiguous() or partials.dim() != 1:
         raise ValueError("fold takes a contiguous 1-D float64 device tensor of partial sums")
     suf, stream = _marshal(out)
-    if out.numel() != 1:
-        raise ValueError("fold writes one element")
+    if out.numel() != 1 or partials.get_device() != out.get_device():
+        raise ValueError("fold writes one element on the device that holds the partial sums")
     _raise(getattr(lib(), f"stream_fold_{suf}")(partials.data_ptr(), out.data_ptr(), 0.0, partials.numel(), stream))
     return out
 
@@ -229,6 +238,8 @@ def shmem_mix(x, out, rounds: int):
         raise ValueError("length or device mismatch")
     if not 0 <= int(rounds) < 2 ** 32:
         raise ValueError("rounds out of range")
+    if x.get_device() != torch.cuda.current_device():
+        raise ValueError("make the tensors' device current around the call")
     stream = torch.cuda.current_stream(x.get_device()).cuda_stream
     _raise(lib().shmem_mix_u32(x.data_ptr(), out.data_ptr(), int(rounds), x.numel(), stream))
     return out
@@ -306,6 +317,11 @@ def check(stream=None):
     import torch
     s = (stream or torch.cuda.current_stream()).cuda_stream
     _raise(lib().streamops_check(s))
+
+
+def set_wait_limit(tries: int):
+    """Attempts a wait inside the bulk-copy pipelines makes before giving up (0 = default)."""
+    _raise(lib().streamops_set_wait_limit(int(tries)))
 
 
 def launch_count() -> int:

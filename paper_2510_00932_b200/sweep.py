@@ -57,44 +57,6 @@ def run(dtypes, iters, sizes=None):
     return rows
 
 
-def run_sequences(n: int = 1 << 25, iters: int = 100):
-    """Call sequences other than the STREAM chain, fp64: microseconds per pass with the automatic
-    traversal direction (the default) and with every kernel walking forwards."""
-    import torch
-    from . import streamops as so
-
-    if not torch.cuda.is_available():
-        raise SystemExit("the sweep needs a CUDA device; there is no CPU fallback")
-    so.lib()
-    so.init(torch.cuda.current_device())
-    a, b, c = (torch.rand(n, dtype=torch.float64, device="cuda") for _ in range(3))
-    seqs = {"copy a->b, copy b->c, copy c->a": lambda: (so.copy(a, b), so.copy(b, c), so.copy(c, a)),
-            "scale a->b, add b+c->a": lambda: (so.scale(a, b, 0.5), so.add(b, c, a)),
-            "triad a+s*b->c, scale c->a, scale a->b": lambda: (so.triad(a, b, c, 0.1), so.scale(c, a, 0.9), so.scale(a, b, 0.9))}
-
-    def time_it(f):
-        for _ in range(5):
-            f()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(iters):
-            f()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / iters * 1e3
-
-    rows = []
-    for name, f in seqs.items():
-        so.reset_tuning()
-        auto = time_it(f)
-        for op in ("copy", "scale", "add", "triad"):
-            so.set_tuning(op, "f64", reverse=0)
-        rows.append({"sequence": name, "n": n, "us_automatic": round(auto, 1), "us_forward": round(time_it(f), 1)})
-        so.reset_tuning()
-    return rows
-
-
 def to_markdown(rows) -> str:
     ops = ("copy", "scale", "add", "triad", "dot")
     out = ["| dtype | n | array | resident | " + " | ".join(f"{o} GB/s" for o in ops) + " |",
@@ -113,12 +75,7 @@ def main(argv=None):
     p.add_argument("--iters", type=int, default=20)
     p.add_argument("--out", default=None)
     p.add_argument("--md", default=None)
-    p.add_argument("--sequences", action="store_true",
-                   help="time other call sequences with the automatic traversal direction and without")
     args = p.parse_args(argv)
-    if args.sequences:
-        print(json.dumps(run_sequences()))
-        return 0
     rows = run(args.dtypes.split(","), args.iters)
     md = to_markdown(rows)
     if args.out:

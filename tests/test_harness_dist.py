@@ -99,3 +99,76 @@ def test_reference_arm_prints_one_json_line():
     r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--workload", "c1",
                         "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=60, env=env)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_launcher_starts_the_ranks_and_rank_zero_prints_one_line(capfd):
+    """The path `bench.py --gpus N` takes when it is started by hand: harness.launch_ranks runs
+    torch.distributed.run with N processes on 127.0.0.1; here N = 2 gloo ranks of a stub."""
+    import json
+    here = os.path.dirname(os.path.abspath(__file__))
+    rc = harness.launch_ranks(os.path.join(here, "rank_stub.py"), ["--steps", "2"], 2)
+    out = capfd.readouterr().out
+    assert rc == 0
+    lines = [l for l in out.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["argv"] == ["--steps", "2"]
+    assert d["ms"] == 15.0 and d["value"] == pytest.approx(3.0e9 / 15e-3 / 1e9)
+
+
+def test_bench_refuses_more_gpus_than_are_visible_and_the_reference_arm_needs_none():
+    import json, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    import torch
+    if torch.cuda.device_count() < 2:
+        r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "1", "--warmup", "1"],
+                           capture_output=True, text=True, timeout=300, env=env)
+        assert r.returncode != 0 and "CUDA device" in r.stderr and "--gpus 2" in r.stderr and r.stdout.strip() == ""
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload", "c1",
+                        "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2
+    # a world size that contradicts --gpus is an error, not a silently mislabelled line
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "4", "--steps", "1"],
+                       capture_output=True, text=True, timeout=300, env=dict(env, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0"))
+    assert r.returncode != 0 and "WORLD_SIZE=2" in r.stderr
+
+
+def test_traffic_summary_round_trip(tmp_path, monkeypatch):
+    """ncu launch list -> per-kernel DRAM bytes of the op-major runs -> what bench.py reads; a
+    capture taken under another tuning is not used."""
+    from paper_2510_00932_b200 import build, ncu_summary
+    build.build()
+    hdr = '"ID","Process ID","Process Name","Host Name","Kernel Name","Context","Stream","Block Size","Grid Size","Device","CC","Section Name","Metric Name","Metric Unit","Metric Value"'
+    add = "void streamops::ew_vec_kernel<double, (int)2, (int)32, (int)2, (int)7>(const T1 *, const T1 *, T1 *, T1, unsigned long, int, int, unsigned long)"
+    cpy = "void streamops::ew_vec_kernel<unsigned long long, (int)0, (int)32, (int)2, (int)7>(const T1 *, const T1 *, T1 *, T1, unsigned long, int, int, unsigned long)"
+    rows, i = [hdr], 0
+
+    def launch(kernel, rd, wr, ns):
+        nonlocal i
+        for m, u, v in (("dram__bytes_read.sum", "Mbyte", rd), ("dram__bytes_write.sum", "Mbyte", wr), ("gpu__time_duration.sum", "ns", ns)):
+            rows.append(f'"{i}","1","python","h","{kernel}","1","7","(128, 1, 1)","(100, 1, 1)","0","10.0","Command line profiler metrics","{m}","{u}","{v}"')
+        i += 1
+
+    for k in (add, cpy, add, cpy):                        # chain-order launches: runs of one, ignored
+        launch(k, 100.0, 100.0, "50,000")
+    for v in (300.0, 536.9, 537.1, 536.8, 537.0):         # op-major run of add (first launch differs)
+        launch(add, v, 268.4, "118,000")
+    for v in (268.4, 268.5, 268.3, 268.4):
+        launch(cpy, v, 268.4, "79,900")
+    p = tmp_path / "l.csv"
+    p.write_text("==PROF== Connected\n" + "\n".join(rows) + "\n")
+    out = tmp_path / "t.txt"
+    assert ncu_summary.main([str(p), "--workload", "c2", "--command", "ncu ...", "--out", str(out)]) == 0
+    data = harness.read_traffic_file(str(out))
+    assert data["kernels"]["add"]["dram_read_bytes"] == 536_950_000 and data["kernels"]["add"]["launch_us"] == 118.0
+    assert data["kernels"]["copy"]["dram_write_bytes"] == 268_400_000 and "dot" not in data["kernels"]
+    monkeypatch.setattr(harness, "traffic_file", lambda w: str(out))
+    from paper_2510_00932_b200 import streamops as so
+    so.reset_tuning()
+    t = so.get_tuning("add", "f64").as_dict()
+    assert harness.captured_traffic("c2", "add", t) == 536_950_000 + 268_400_000
+    assert harness.captured_traffic("c2", "add", dict(t, unroll=4)) is None
+    assert harness.captured_traffic("c2", "dot", so.get_tuning("dot", "f64").as_dict()) is None
