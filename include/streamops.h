@@ -221,14 +221,21 @@ typedef struct streamops_tuning {
     int pdl;            /* kind 0: 1 = programmatic dependent launch: the kernel's blocks may become
                            resident while the previous kernel of the stream drains, and wait inside
                            the kernel until it has completed (hides launch latency) */
-    int keep_mib;       /* kind 0, policies 7 and 8: the last keep_mib MiB of output in traversal order are
+    int keep_mib;       /* kind 0, policies 7 and 8, in a call one of whose inputs is the array the previous
+                           elementwise call on the device wrote (a link of a dataflow chain, whose own output
+                           is likely to be read next): the last keep_mib MiB of output in traversal order are
                            stored plainly (7) or with evict_last L2 priority (8) and are what the kernel
                            leaves in L2 for its consumer; everything before is stored evict_first, so that
-                           the kernel's own output does not push out the lines its producer left there */
+                           the kernel's own output does not push out the lines its producer left there. In
+                           any other call policies 7 and 8 store evict_first throughout, as policy 4 */
     int compensated;    /* Dot, kind 0: 1 = carry every accumulator as a (sum, error) pair (two-sum and, for
                            double inputs, an exact product split: the published Dot2 scheme): the result is
                            as accurate as a sum done in about twice the working precision, for inputs whose
                            dot product cancels heavily; ~10 double operations per element instead of one */
+    int pipeline;       /* Dot, kind 0, 32-byte vectors: 1 = rolling-slot kernel: a thread keeps `unroll` (2 or 4)
+                           slots of one vector per array, folds the oldest into its accumulator and reloads it
+                           at once, so that loads stay in flight all the time; 0 = a tile of `unroll` vectors per
+                           array is requested, awaited and folded as a whole */
 } streamops_tuning_t;
 
 int streamops_set_tuning(int op, int dtype, const streamops_tuning_t *t);

@@ -18,9 +18,9 @@ constexpr int kChainRing = 4;           // stages of the host-buffer pipeline: p
 // One Dot workspace slot of a device. A slot belongs to the stream that used it last: that stream
 // may use it again at once (its Dots run in stream order); another stream may take it over only
 // when the slot's last Dot has finished. Every Dot gets the next sequence number of its slot
-// (`issued`), and the kernel that finishes it writes that number to the slot's word of the device
-// array `done_seq` as its last act: the slot is idle when the two agree. Nothing is added to the
-// stream between kernels (an event record there would end the overlap of dependent launches).
+// (`issued`), and the block that finishes it writes that number into the high half of the slot's
+// ticket word as its last act: the slot is idle when the two agree. Nothing is added to the stream
+// between kernels (an event record there would end the overlap of dependent launches).
 struct DotSlot {
     cudaStream_t owner = nullptr;
     unsigned issued = 0;
@@ -31,10 +31,9 @@ struct DeviceState {
     std::atomic<bool> ready{false};
     int sm_count = 0;
     double *partials = nullptr;        // kDotSlots * kMaxDotBlocks doubles
-    unsigned *tickets = nullptr;       // kDotSlots counters, zero between calls
+    unsigned long long *tickets = nullptr;   // kDotSlots ticket words (see DotScratch), low halves zero between calls
     int *error_flag = nullptr;         // set by a bounded wait that gave up
-    unsigned *done_seq = nullptr;      // kDotLiveSlots words, see DotSlot
-    unsigned *done_host = nullptr;     // pinned host copy, refreshed only when a slot has to change hands
+    unsigned long long *done_host = nullptr;   // pinned host copy of the ticket words, refreshed only when a slot has to change hands
     cudaStream_t probe_stream = nullptr;   // carries that refresh, so that no caller's stream is touched
     std::mutex slot_mutex;
     DotSlot slots[kDotLiveSlots];      // slots of ordinary calls; the rest serve stream capture
@@ -77,16 +76,20 @@ std::atomic<unsigned long long> g_launches{0};
 streamops_tuning_t default_tuning(int op, int dtype) {
     streamops_tuning_t t;
     t.kind = 0; t.vec_bytes = 32; t.unroll = 2; t.threads = 256; t.blocks_per_sm = 0;
-    t.policy = 7; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0; t.reverse = 0; t.pdl = 1; t.keep_mib = 112; t.compensated = 0;
+    t.policy = 7; t.contiguous = 0; t.chunk_bytes = 16384; t.stages = 4; t.two_pass = 0; t.reverse = 0; t.pdl = 1; t.keep_mib = 112; t.compensated = 0; t.pipeline = 0;
     const bool f64 = dtype == DT_F64;
     switch (op) {
         case OP_COPY:  t.reverse = 2; break;
         case OP_SCALE: t.reverse = 2; break;
         case OP_ADD:   t.threads = 128; t.reverse = 2; break;
         case OP_TRIAD: t.threads = 128; t.reverse = 2; break;
-        // Dot, double: persistent grid sized automatically (blocks_per_sm = 0: 2 or 3 per SM, see
-        // resolve_vec); float: 2 per SM and two vectors in flight measured best from 16 MiB to 2 GiB
-        case OP_DOT:   t.threads = 512; t.policy = 4; t.unroll = f64 ? 4 : 2; t.blocks_per_sm = f64 ? 0 : 2; break;
+        // Dot, double: the rolling-slot kernel with two slots per thread on two blocks per SM (measured
+        // against the tile-at-a-time kernel: 77.4 vs 78.4 us at n = 2^25, equal at 2^28, 9.7 vs 12.4 us at
+        // 2^22); float: tiles of two vectors on two blocks per SM measured best from 16 MiB to 2 GiB
+        case OP_DOT:
+            t.threads = 512; t.policy = 4; t.unroll = 2;
+            t.pipeline = f64 ? 1 : 0; t.blocks_per_sm = f64 ? 0 : 2;
+            break;
     }
     return t;
 }
@@ -114,10 +117,10 @@ int cuda_fail(cudaError_t e) {
 }
 
 void free_workspace(DeviceState &d) {
-    cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag); cudaFree(d.done_seq);
+    cudaFree(d.partials); cudaFree(d.tickets); cudaFree(d.error_flag);
     if (d.done_host) cudaFreeHost(d.done_host);
     if (d.probe_stream) cudaStreamDestroy(d.probe_stream);
-    d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr; d.done_seq = nullptr;
+    d.partials = nullptr; d.tickets = nullptr; d.error_flag = nullptr;
     d.done_host = nullptr; d.probe_stream = nullptr;
     for (DotSlot &s : d.slots) s = DotSlot{};
 }
@@ -137,16 +140,14 @@ int init_device(int device, DeviceState **out) {
                 if ((e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { status = cuda_fail(e); break; }
                 const size_t pbytes = sizeof(double) * kDotSlots * kMaxDotBlocks;
                 if (cudaMalloc(&d.partials, pbytes) != cudaSuccess ||
-                    cudaMalloc(&d.tickets, sizeof(unsigned) * kDotSlots) != cudaSuccess ||
+                    cudaMalloc(&d.tickets, sizeof(unsigned long long) * kDotSlots) != cudaSuccess ||
                     cudaMalloc(&d.error_flag, sizeof(int)) != cudaSuccess ||
-                    cudaMalloc(&d.done_seq, sizeof(unsigned) * kDotLiveSlots) != cudaSuccess ||
-                    cudaMallocHost(&d.done_host, sizeof(unsigned) * kDotLiveSlots) != cudaSuccess) {
+                    cudaMallocHost(&d.done_host, sizeof(unsigned long long) * kDotLiveSlots) != cudaSuccess) {
                     (void)cudaGetLastError();
                     status = STREAMOPS_ERR_WORKSPACE; break;
                 }
-                if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned) * kDotSlots)) != cudaSuccess) { status = cuda_fail(e); break; }
+                if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned long long) * kDotSlots)) != cudaSuccess) { status = cuda_fail(e); break; }
                 if ((e = cudaMemset(d.error_flag, 0, sizeof(int))) != cudaSuccess) { status = cuda_fail(e); break; }
-                if ((e = cudaMemset(d.done_seq, 0, sizeof(unsigned) * kDotLiveSlots)) != cudaSuccess) { status = cuda_fail(e); break; }
                 if ((e = cudaStreamCreateWithFlags(&d.probe_stream, cudaStreamNonBlocking)) != cudaSuccess) { status = cuda_fail(e); break; }
                 for (DotSlot &s : d.slots) s = DotSlot{};
             } while (false);
@@ -213,14 +214,17 @@ VecLaunch resolve_vec(const streamops_tuning_t &t, const DeviceState &d, int op,
     c.contiguous = t.contiguous;
     c.reverse = t.reverse == 1;                                  // 2 (automatic) is resolved by the caller
     c.pdl = t.pdl != 0;
+    c.pipeline = (op == OP_DOT && t.pipeline && c.vec_bytes == 32 && c.unroll >= 2) ? 1 : 0;
     c.policy = t.policy;
     // the read-only data path must not be used on an array the kernel also writes
     if (c.policy == 1 && (out == x || out == y)) c.policy = 0;
     if (op == OP_DOT && c.policy > 6) c.policy = 4;           // Dot stores nothing: the two-phase sets reduce to 4
-    const size_t per_tile = (size_t)c.threads * (c.vec_bytes ? (size_t)c.unroll * c.vec_bytes / esize : 1);
+    const size_t per_tile = (size_t)c.threads * (c.vec_bytes ? (size_t)(c.pipeline ? 1 : c.unroll) * c.vec_bytes / esize : 1);
     const size_t tiles = (n + per_tile - 1) / per_tile;
     size_t grid = t.blocks_per_sm > 0 ? (size_t)t.blocks_per_sm * d.sm_count : tiles;
-    if (op == OP_DOT && t.blocks_per_sm == 0) {
+    if (op == OP_DOT && t.blocks_per_sm == 0 && c.pipeline) {
+        grid = (size_t)2 * d.sm_count;                           // the rolling-slot kernel keeps two blocks per SM busy
+    } else if (op == OP_DOT && t.blocks_per_sm == 0) {
         // automatic persistent grid: a third block per SM (which starts as the first two finish and
         // evens out the tail) pays once every block has several tiles; small arrays do best with two
         const size_t three = (size_t)3 * d.sm_count;
@@ -243,6 +247,7 @@ bool valid_tuning(const streamops_tuning_t &t) {
     if (t.policy < 0 || t.policy > 8) return false;
     if (t.keep_mib < 0 || t.keep_mib > 65536) return false;
     if (t.compensated != 0 && t.compensated != 1) return false;
+    if (t.pipeline != 0 && t.pipeline != 1) return false;
     if (t.chunk_bytes < 1024 || t.chunk_bytes > 65536 || (t.chunk_bytes & 15)) return false;
     if (t.stages < 2 || t.stages > 8) return false;
     if (t.reverse < 0 || t.reverse > 2) return false;
@@ -251,9 +256,8 @@ bool valid_tuning(const streamops_tuning_t &t) {
 
 // Picks the workspace slot of one Dot call on `stream` and fills in its scratch pointers.
 // Ordinary calls: the slot this stream used last (stream order makes reuse safe), else a slot never
-// used, else a slot whose last Dot has finished (the device's done_seq words are copied to the host
-// on a stream of the library's own: this is the only path that waits for anything, and only for
-// that copy); if all kDotLiveSlots slots are still in flight on other streams, STREAMOPS_ERR_WORKSPACE.
+// used, else a slot whose last Dot has finished (the ticket words are copied to the host on a stream
+// of the library's own: this is the only path that waits for anything, and only for that copy); if all kDotLiveSlots slots are still in flight on other streams, STREAMOPS_ERR_WORKSPACE.
 // Calls made while `stream` is being captured: one of the kDotCaptureSlots slots set aside for graphs,
 // handed out in turn and never shared with ordinary calls; the slot is baked into the graph.
 int acquire_dot_slot(DeviceState *d, cudaStream_t stream, DotScratch *scratch, DotSlot **live) {
@@ -264,7 +268,6 @@ int acquire_dot_slot(DeviceState *d, cudaStream_t stream, DotScratch *scratch, D
     int found = -1;
     if (capturing != cudaStreamCaptureStatusNone) {
         found = kDotLiveSlots + (int)(d->next_capture_slot.fetch_add(1) % (unsigned)kDotCaptureSlots);
-        scratch->done = nullptr;
         scratch->seq = 0;
     } else {
         std::lock_guard<std::mutex> lock(d->slot_mutex);
@@ -273,19 +276,19 @@ int acquire_dot_slot(DeviceState *d, cudaStream_t stream, DotScratch *scratch, D
         for (int i = 0; i < kDotLiveSlots && found < 0; ++i)
             if (!d->slots[i].used) found = i;
         if (found < 0) {
-            if ((e = cudaMemcpyAsync(d->done_host, d->done_seq, sizeof(unsigned) * kDotLiveSlots, cudaMemcpyDeviceToHost,
+            if ((e = cudaMemcpyAsync(d->done_host, d->tickets, sizeof(unsigned long long) * kDotLiveSlots, cudaMemcpyDeviceToHost,
                                      d->probe_stream)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaStreamSynchronize(d->probe_stream)) != cudaSuccess) return cuda_fail(e);
             for (int k = 0; k < kDotLiveSlots && found < 0; ++k) {
                 const int i = (int)((d->steal_cursor + (unsigned)k) % (unsigned)kDotLiveSlots);
-                if (d->done_host[i] == d->slots[i].issued) { found = i; d->steal_cursor = (unsigned)i + 1; }
+                // finished: the high half carries the last issued number (and the ticket is back at zero)
+                if (d->done_host[i] == ((unsigned long long)d->slots[i].issued << 32)) { found = i; d->steal_cursor = (unsigned)i + 1; }
             }
         }
         if (found < 0) return STREAMOPS_ERR_WORKSPACE;
         DotSlot &s = d->slots[found];
         s.used = true;
         s.owner = stream;
-        scratch->done = d->done_seq + found;
         scratch->seq = ++s.issued;
         *live = &s;
     }
@@ -311,7 +314,7 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
     if ((status = current_device_state(&d)) != STREAMOPS_OK) return status;
     const streamops_tuning_t t = tuning(op, dtype);
 
-    DotScratch scratch{nullptr, nullptr, nullptr, 0};
+    DotScratch scratch{nullptr, nullptr, 0};
     DotSlot *live_slot = nullptr;
     if (op == OP_DOT && (status = acquire_dot_slot(d, stream, &scratch, &live_slot)) != STREAMOPS_OK) return status;
 
@@ -335,14 +338,18 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
     } else {
         VecLaunch c = resolve_vec(t, *d, op, esize, x, y, out, n);
         if (op != OP_DOT) {
-            if (t.reverse == 2) {
-                // automatic direction: if an input is the array the previous elementwise kernel wrote,
-                // start at the end that kernel wrote last (its lines are the ones still in L2)
-                const uintptr_t w = d->last_written.load();
-                const bool consumer = w != 0 && d->last_written_bytes.load() == n * esize &&
-                                      (w == (uintptr_t)x || (uses_y && w == (uintptr_t)y));
-                c.reverse = consumer && d->last_written_end_high.load() != 0;
-            }
+            // is an input of this call the array the previous elementwise kernel on the device wrote?
+            const uintptr_t w = d->last_written.load();
+            const bool consumer = w != 0 && d->last_written_bytes.load() == n * esize &&
+                                  (w == (uintptr_t)x || (uses_y && w == (uintptr_t)y));
+            // automatic direction: a consumer starts at the end its producer wrote last (those lines are
+            // the ones still in L2)
+            if (t.reverse == 2) c.reverse = consumer && d->last_written_end_high.load() != 0;
+            // two-phase stores keep the end of the output in L2 for a consumer. A call that is itself a
+            // consumer is a link of a dataflow chain, so its output is likely to be read next; a call
+            // that is not gets streaming (evict-first) stores throughout, which is the faster choice
+            // when nobody comes for the output
+            if ((c.policy == 7 || c.policy == 8) && !consumer) c.policy = 4;
             d->last_written.store((uintptr_t)out);
             d->last_written_bytes.store(n * esize);
             d->last_written_end_high.store(c.reverse ? 0 : 1);       // a forward walk finishes at the high end
@@ -609,8 +616,8 @@ const char *streamops_policy_name(int policy) {
         case 4: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first";
         case 5: return "ld.global.L1::no_allocate + L2 evict_first / st.global";
         case 6: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_last";
-        case 7: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, plain st.global for the last keep_mib MiB";
-        case 8: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, evict_last for the last keep_mib MiB";
+        case 7: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, plain st.global for the last keep_mib MiB when the call consumes the previous call's output";
+        case 8: return "ld.global.L1::no_allocate + L2 evict_first / st.global + L2 evict_first, evict_last for the last keep_mib MiB when the call consumes the previous call's output";
         default: return "unknown";
     }
 }

@@ -209,8 +209,7 @@ __device__ __forceinline__ T apply(T x, T y, T s) {
 template <typename T, int OP, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads + 32)
 bulk_compute_kernel(const T *x, const T *y, T *out, T s, size_t n, unsigned chunk, int stages,
-                    double *partials, unsigned *ticket, int *error_flag, unsigned wait_limit,
-                    unsigned *done, unsigned seq) {
+                    double *partials, unsigned long long *ticket, int *error_flag, unsigned wait_limit, unsigned seq) {
     constexpr bool USES_Y = (OP != OP_SCALE);
     constexpr int EPV = 16 / (int)sizeof(T);
     extern __shared__ __align__(128) unsigned char smem[];
@@ -286,7 +285,7 @@ bulk_compute_kernel(const T *x, const T *y, T *out, T s, size_t n, unsigned chun
     }
     if constexpr (OP == OP_DOT) {
         const double bsum = block_sum(acc, warp_part);
-        publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, done, seq);
+        publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, seq);
     }
 }
 
@@ -303,7 +302,7 @@ cudaError_t launch_compute(const BulkLaunch &c, const T *x, const T *y, T *out, 
     cudaError_t e = allow_smem(kernel, smem);
     if (e != cudaSuccess) return e;
     kernel<<<c.grid, c.threads + 32, smem, st>>>(x, y, out, (T)scalar, n, (unsigned)c.chunk_bytes, c.stages,
-                                                 sc.partials, sc.ticket, error_flag, c.wait_limit, sc.done, sc.seq);
+                                                 sc.partials, sc.ticket, error_flag, c.wait_limit, sc.seq);
     return cudaGetLastError();
 }
 

@@ -6,6 +6,12 @@
 // folded in a fixed order: per thread (u = 0..U-1), per warp (xor-shuffle tree), per block
 // (shared memory, warp 0 folds the warp sums), giving partials[blockIdx.x].
 //
+// A second pass-1 form, the rolling-slot kernel, gives each thread S slots of one vector of x and one
+// of y: the oldest slot is folded into its accumulator and reloaded at once, so S - 1 loads per array
+// stay in flight per thread all the time instead of all of them draining before the next tile is
+// requested. Slot s of thread t owns tiles b + (s + k S) G (k = 0, 1, ...) of block b: still a fixed
+// function of n and the launch shape.
+//
 // Pass 2 sums partials[0..G-1] with one block in a fixed order (thread t takes t, t + B, ... in
 // sequence, then the same warp/block tree). It runs either as its own launch or inside pass 1
 // by whichever block arrives last at an atomic ticket: the ticket only elects WHO does pass 2,
@@ -30,8 +36,8 @@ __device__ __forceinline__ double fold_vec(double acc, const Vec<VB> &xv, const 
 
 template <typename T, int VB, int U, int POL, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads)
-dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int reverse,
-                 unsigned *done, unsigned seq) {
+dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned long long *ticket, T *out, int reverse,
+                 unsigned seq) {
     constexpr int EPV = VB / (int)sizeof(T);
     __shared__ double warp_part[32];
     __shared__ bool is_last;
@@ -72,22 +78,87 @@ dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *t
     for (int u = 1; u < U; ++u) tsum += acc[u];
     const double bsum = block_sum(tsum, warp_part);
 
-    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, done, seq);
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, seq);
+}
+
+// Rolling-slot pass 1 (see the file comment). A tile is blockDim.x vectors: one vector per thread.
+template <typename T, int VB, int S, int POL, bool SINGLE_LAUNCH>
+__global__ void __launch_bounds__(kMaxThreads, S <= 2 ? 2 : 1)
+dot_roll_kernel(const T *x, const T *y, size_t n, double *partials, unsigned long long *ticket, T *out, unsigned seq) {
+    constexpr int EPV = VB / (int)sizeof(T);
+    __shared__ double warp_part[32];
+    __shared__ bool is_last;
+    grid_dependency_sync();
+    const char *xb = reinterpret_cast<const char *>(x);
+    const char *yb = reinterpret_cast<const char *>(y);
+    const uint64_t l2pol = make_l2_policies<POL>().ld;
+
+    const size_t nvec = n / EPV;
+    const size_t ntiles = nvec / blockDim.x;
+    const size_t G = gridDim.x;
+    // byte offsets: a slot's vector of tile k sits at k * tile_bytes + threadIdx.x * VB, so "tile k exists"
+    // is "offset < end"; slots of one round are slot_stride apart, rounds are round_stride apart
+    const size_t tile_bytes = (size_t)blockDim.x * VB;
+    const size_t end = ntiles * tile_bytes;
+    const size_t slot_stride = G * tile_bytes;
+    const size_t round_stride = (size_t)S * slot_stride;
+    size_t off = (size_t)blockIdx.x * tile_bytes + (size_t)threadIdx.x * VB;
+    double acc[S];
+    Vec<VB> xv[S], yv[S];
+#pragma unroll
+    for (int s = 0; s < S; ++s) acc[s] = 0.0;
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+        const size_t o = off + (size_t)s * slot_stride;
+        if (o < end) {
+            ldg<POL>(xv[s], xb + o, l2pol);
+            ldg<POL>(yv[s], yb + o, l2pol);
+        }
+    }
+    for (; off < end; off += round_stride) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+            const size_t o = off + (size_t)s * slot_stride;
+            if (o < end) {
+                acc[s] = fold_vec<T, VB>(acc[s], xv[s], yv[s]);
+                const size_t next = o + round_stride;
+                if (next < end) {
+                    ldg<POL>(xv[s], xb + next, l2pol);
+                    ldg<POL>(yv[s], yb + next, l2pol);
+                }
+            }
+        }
+    }
+    if (blockIdx.x == (unsigned)(ntiles % G)) {              // ragged end, one block
+        for (size_t v = ntiles * blockDim.x + threadIdx.x; v < nvec; v += blockDim.x) {
+            Vec<VB> xr, yr;
+            ldg<0>(xr, xb + v * VB, 0);
+            ldg<0>(yr, yb + v * VB, 0);
+            acc[0] = fold_vec<T, VB>(acc[0], xr, yr);
+        }
+        const size_t i = nvec * EPV + threadIdx.x;
+        if (i < n) acc[0] = fma(widen<T>(x[i]), widen<T>(y[i]), acc[0]);
+    }
+    double tsum = acc[0];
+#pragma unroll
+    for (int s = 1; s < S; ++s) tsum += acc[s];
+    const double bsum = block_sum(tsum, warp_part);
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, seq);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(1024)
-dot_pass2_kernel(const double *partials, unsigned count, T *out, unsigned *done, unsigned seq) {
+dot_pass2_kernel(const double *partials, unsigned count, T *out, unsigned long long *ticket, unsigned seq) {
     __shared__ double warp_part[32];
     finish<T>(partials, count, out, warp_part);
-    if (threadIdx.x == 0) mark_done(done, seq);
+    if (threadIdx.x == 0) rearm(ticket, seq);
 }
 
 // Scalar pass 1 for pointers that are not 16-byte aligned: same structure, one element per load.
 template <typename T, bool SINGLE_LAUNCH>
 __global__ void __launch_bounds__(kMaxThreads)
-dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out,
-                  unsigned *done, unsigned seq) {
+dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned long long *ticket, T *out,
+                  unsigned seq) {
     __shared__ double warp_part[32];
     __shared__ bool is_last;
     double acc = 0.0;
@@ -95,18 +166,29 @@ dot_scalar_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
         acc = fma(widen<T>(x[i]), widen<T>(y[i]), acc);
     const double bsum = block_sum(acc, warp_part);
-    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, done, seq);
+    publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, seq);
 }
 
 template <typename T, int VB, int U, bool SL>
 cudaError_t launch_pol(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
     switch (c.policy) {
-#define STREAMOPS_CASE(P) case P: return launch_kernel(dot_pass1_kernel<T, VB, U, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, c.reverse, s.done, s.seq);
+#define STREAMOPS_CASE(P) case P: return launch_kernel(dot_pass1_kernel<T, VB, U, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, c.reverse, s.seq);
         STREAMOPS_CASE(0) STREAMOPS_CASE(1) STREAMOPS_CASE(2) STREAMOPS_CASE(3) STREAMOPS_CASE(4) STREAMOPS_CASE(5) STREAMOPS_CASE(6)
 #undef STREAMOPS_CASE
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
+}
+
+// The rolling-slot kernel loads with the evict-first set (4) or with plain loads (0).
+template <typename T, int VB, bool SL>
+cudaError_t launch_roll(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
+    const bool plain = c.policy == 0;
+#define STREAMOPS_ROLL(S, P) launch_kernel(dot_roll_kernel<T, VB, S, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, s.seq)
+    if (c.unroll == 2) return plain ? STREAMOPS_ROLL(2, 0) : STREAMOPS_ROLL(2, 4);
+    if (c.unroll == 4) return plain ? STREAMOPS_ROLL(4, 0) : STREAMOPS_ROLL(4, 4);
+#undef STREAMOPS_ROLL
+    return cudaErrorInvalidValue;
 }
 
 template <typename T, int VB, bool SL>
@@ -121,9 +203,10 @@ cudaError_t launch_unroll(const VecLaunch &c, const T *x, const T *y, size_t n, 
 
 template <typename T, bool SL>
 cudaError_t launch_pass1(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
+    if (c.vec_bytes == 32 && c.pipeline) return launch_roll<T, 32, SL>(c, x, y, n, s, out, st);
     if (c.vec_bytes == 32) return launch_unroll<T, 32, SL>(c, x, y, n, s, out, st);
     if (c.vec_bytes == 16) return launch_unroll<T, 16, SL>(c, x, y, n, s, out, st);
-    dot_scalar_kernel<T, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out, s.done, s.seq);
+    dot_scalar_kernel<T, SL><<<c.grid, c.threads, 0, st>>>(x, y, n, s.partials, s.ticket, out, s.seq);
     return cudaGetLastError();
 }
 
@@ -143,7 +226,7 @@ cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, bool wide, const T *
         *launches = 2;
         cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, (T *)nullptr, st);
         if (e != cudaSuccess) return e;
-        dot_pass2_kernel<double><<<1, 1024, 0, st>>>(s.partials, c.grid, (double *)out, s.done, s.seq);
+        dot_pass2_kernel<double><<<1, 1024, 0, st>>>(s.partials, c.grid, (double *)out, s.ticket, s.seq);
         return cudaGetLastError();
     }
     T *o = (T *)out;
@@ -154,7 +237,7 @@ cudaError_t launch_dot_t(const VecLaunch &c, bool two_pass, bool wide, const T *
     *launches = 2;
     cudaError_t e = launch_pass1<T, false>(c, x, y, n, s, o, st);
     if (e != cudaSuccess) return e;
-    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, o, s.done, s.seq);
+    dot_pass2_kernel<T><<<1, 1024, 0, st>>>(s.partials, c.grid, o, s.ticket, s.seq);
     return cudaGetLastError();
 }
 

@@ -73,8 +73,8 @@ __device__ __forceinline__ Pair block_merge(Pair v, Pair *warp_part) {
 
 template <typename T, int U>
 __global__ void __launch_bounds__(kMaxThreads, 2)
-dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ticket, T *out, int vectorised,
-                unsigned *done, unsigned seq) {
+dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned long long *ticket, T *out, int vectorised,
+                unsigned seq) {
     constexpr int EPV = 32 / (int)sizeof(T);
     __shared__ Pair warp_part[32];
     __shared__ bool is_last;
@@ -121,12 +121,10 @@ dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ti
     if (threadIdx.x == 0) {
         partials[2 * blockIdx.x] = b.s;
         partials[2 * blockIdx.x + 1] = b.c;
-        __threadfence();                                          // pair visible before the ticket
-        is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+        is_last = arrive(ticket) == gridDim.x - 1;                // releases the pair, acquires the others'
     }
     __syncthreads();
     if (is_last) {                                                // fixed-order merge of all blocks' pairs
-        __threadfence();
         Pair a{0.0, 0.0};
         for (unsigned k = threadIdx.x; k < gridDim.x; k += blockDim.x)
             a = merge(a, Pair{__ldcg(partials + 2 * k), __ldcg(partials + 2 * k + 1)});
@@ -134,8 +132,7 @@ dot_comp_kernel(const T *x, const T *y, size_t n, double *partials, unsigned *ti
         const Pair total = block_merge(a, warp_part);
         if (threadIdx.x == 0) {
             out[0] = (T)__dadd_rn(total.s, total.c);
-            *ticket = 0u;
-            mark_done(done, seq);
+            rearm(ticket, seq);
         }
     }
 }
@@ -144,9 +141,9 @@ template <typename T>
 cudaError_t launch_t(const VecLaunch &c, const T *x, const T *y, T *out, size_t n, const DotScratch &s, cudaStream_t st) {
     const int vec = c.vec_bytes == 32;
     switch (vec ? c.unroll : 1) {
-        case 1: return launch_kernel(dot_comp_kernel<T, 1>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.done, s.seq);
-        case 2: return launch_kernel(dot_comp_kernel<T, 2>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.done, s.seq);
-        case 4: return launch_kernel(dot_comp_kernel<T, 4>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.done, s.seq);
+        case 1: return launch_kernel(dot_comp_kernel<T, 1>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.seq);
+        case 2: return launch_kernel(dot_comp_kernel<T, 2>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.seq);
+        case 4: return launch_kernel(dot_comp_kernel<T, 4>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, vec, s.seq);
         default: return cudaErrorInvalidValue;
     }
 }

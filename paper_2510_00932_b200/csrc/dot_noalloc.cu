@@ -43,7 +43,7 @@ dot_noalloc_kernel(const double *x, const double *y, size_t n, double *scratch, 
     __shared__ double warp_part[32];
     __shared__ bool is_last;
     double *partials = scratch;
-    unsigned *ticket = reinterpret_cast<unsigned *>(scratch + kTicketSlot);
+    unsigned long long *ticket = reinterpret_cast<unsigned long long *>(scratch + kTicketSlot);
 
     const size_t begin = (size_t)blockIdx.x * kSpan;
     const size_t len = n - begin < kSpan ? n - begin : kSpan;
@@ -79,7 +79,7 @@ dot_noalloc_kernel(const double *x, const double *y, size_t n, double *scratch, 
     }
     const double tsum = ((acc[0] + acc[1]) + acc[2]) + acc[3];
     const double bsum = block_sum(tsum, warp_part);
-    publish_partial<double, true>(bsum, partials, ticket, out, warp_part, &is_last, nullptr, 0u);
+    publish_partial<double, true>(bsum, partials, ticket, out, warp_part, &is_last, 0u);
 }
 
 // Device address of the scratch array, looked up once per device with that device current.
@@ -125,7 +125,7 @@ extern "C" int stream_dot_noalloc_f64(const double *x, const double *y, double *
     if ((e = scratch_for_current_device(&scratch)) != cudaSuccess) return note_cuda_error(e);
     // the array keeps the last call's contents: the ticket must start at zero (an interrupted
     // earlier call could have left it mid-count); the partial sums are all rewritten before use
-    if ((e = cudaMemsetAsync(scratch + kTicketSlot, 0, sizeof(unsigned), stream)) != cudaSuccess) return note_cuda_error(e);
+    if ((e = cudaMemsetAsync(scratch + kTicketSlot, 0, sizeof(unsigned long long), stream)) != cudaSuccess) return note_cuda_error(e);
     const unsigned blocks = (unsigned)((n + kSpan - 1) / kSpan);
     const int vectorised = (((uintptr_t)x | (uintptr_t)y) & 31) == 0;
     dot_noalloc_kernel<<<blocks, kThreads, 0, stream>>>(x, y, n, scratch, out, vectorised);

@@ -25,6 +25,7 @@ struct VecLaunch {
     int contiguous;
     int reverse;       // 1 = walk the tiles from the high addresses down
     int pdl;           // 1 = launch with programmatic stream serialization
+    int pipeline;      // Dot: 1 = rolling-slot kernel (unroll = slots per thread)
     size_t hot_tiles;  // policies 7, 8: tiles at the start of the traversal whose stores are evict-first
 };
 
@@ -69,10 +70,14 @@ __device__ __forceinline__ void grid_dependency_sync() {
 // Per-slot Dot scratch: partial sums written by pass 1, the arrival ticket of the single-launch
 // variant, and (shared) the device error flag.
 struct DotScratch {
-    double *partials;      // kMaxDotBlocks doubles
-    unsigned *ticket;      // one counter, zero between calls
-    unsigned *done;        // where the kernel that finishes the Dot writes `seq` as its last act (may be null)
-    unsigned seq;          // this call's sequence number on its slot
+    double *partials;              // kMaxDotBlocks doubles
+    // One 64-bit word per slot. Low half: the arrival ticket, zero between calls (blocks add to it
+    // through a 32-bit pointer to the word's first four bytes). High half: the sequence number of the
+    // last Dot that FINISHED on the slot. The block that finishes a Dot writes the whole word with one
+    // store -- (seq << 32) | 0 -- after its last read of the partial sums, which re-arms the ticket and
+    // tells the host, when it needs to know, that the slot is free.
+    unsigned long long *ticket;
+    unsigned seq;                  // this call's sequence number on its slot (0 for slots used by graphs)
 };
 
 // api.cu: bookkeeping shared by the entry points that live in other files

@@ -28,46 +28,43 @@ __device__ __forceinline__ double block_sum(double v, double *warp_part) {
 
 template <typename T> __device__ __forceinline__ double widen(T v) { return (double)v; }
 
-// Fixed-order sum of partials[0..count-1] by one block; thread 0 writes (T)total to out.
+// Fixed-order sum of partials[0..count-1] by one block; thread 0 writes (T)total to out. The caller
+// makes sure (with a barrier) that nobody is still reading warp_part from an earlier block_sum.
 template <typename T>
 __device__ __forceinline__ void finish(const double *partials, unsigned count, T *out, double *warp_part) {
     double acc = 0.0;
     for (unsigned b = threadIdx.x; b < count; b += blockDim.x) acc += __ldcg(partials + b);
-    __syncthreads();                      // warp_part is reused
     const double total = block_sum(acc, warp_part);
     if (threadIdx.x == 0) out[0] = (T)total;
 }
 
-// Last act of the thread that finishes a Dot: after everything it read or wrote in the slot's
-// scratch, it publishes the call's sequence number, which tells the host (when it needs to know)
-// that the slot is free for another stream.
-__device__ __forceinline__ void mark_done(unsigned *done, unsigned seq) {
-    if (done) {
-        __threadfence();
-        *done = seq;
-    }
+// Arrival at a slot's ticket: one atomic add with release and acquire semantics. The release half
+// publishes the partial sum this thread stored just before; the acquire half of the LAST arrival
+// makes every earlier block's partial sum visible to it (the adds form one release sequence), so no
+// separate fences are needed.
+__device__ __forceinline__ unsigned arrive(unsigned long long *ticket_word) {
+    unsigned t;
+    asm volatile("atom.add.acq_rel.gpu.u32 %0, [%1], 1;" : "=r"(t) : "l"(ticket_word) : "memory");
+    return t;
+}
+// Last act of the block that finishes a Dot: ticket back to zero and the call's sequence number in the
+// word's high half, in one store (see DotScratch).
+__device__ __forceinline__ void rearm(unsigned long long *ticket_word, unsigned seq) {
+    *ticket_word = (unsigned long long)seq << 32;
 }
 
 // Publishes this block's partial sum; in the single-launch form the block that arrives last at
 // the ticket then folds all partials (in block-index order) and re-arms the ticket.
 template <typename T, bool SINGLE_LAUNCH>
-__device__ __forceinline__ void publish_partial(double bsum, double *partials, unsigned *ticket, T *out,
-                                                double *warp_part, bool *is_last, unsigned *done, unsigned seq) {
+__device__ __forceinline__ void publish_partial(double bsum, double *partials, unsigned long long *ticket, T *out,
+                                                double *warp_part, bool *is_last, unsigned seq) {
     if (threadIdx.x == 0) partials[blockIdx.x] = bsum;
     if constexpr (SINGLE_LAUNCH) {
-        if (threadIdx.x == 0) {
-            __threadfence();                                  // partial visible before the ticket
-            const unsigned t = atomicAdd(ticket, 1u);
-            *is_last = (t == gridDim.x - 1);
-        }
+        if (threadIdx.x == 0) *is_last = (arrive(ticket) == gridDim.x - 1);
         __syncthreads();
         if (*is_last) {
-            __threadfence();
             finish<T>(partials, gridDim.x, out, warp_part);
-            if (threadIdx.x == 0) {
-                *ticket = 0u;                                 // ready for the next call
-                mark_done(done, seq);
-            }
+            if (threadIdx.x == 0) rearm(ticket, seq);
         }
     }
 }

@@ -31,7 +31,7 @@ class Tuning(ctypes.Structure):
     """Mirror of streamops_tuning_t."""
     _fields_ = [(n, ctypes.c_int) for n in (
         "kind", "vec_bytes", "unroll", "threads", "blocks_per_sm", "policy", "contiguous",
-        "chunk_bytes", "stages", "two_pass", "reverse", "pdl", "keep_mib", "compensated")]
+        "chunk_bytes", "stages", "two_pass", "reverse", "pdl", "keep_mib", "compensated", "pipeline")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

@@ -47,6 +47,10 @@ VEC_TUNINGS = [
     dict(kind=0, vec_bytes=16, unroll=4, threads=256, blocks_per_sm=3, policy=6, contiguous=1, reverse=1),
     dict(kind=0, vec_bytes=32, unroll=4, threads=256, blocks_per_sm=0, policy=7, contiguous=0, reverse=0, keep_mib=1),
     dict(kind=0, vec_bytes=16, unroll=2, threads=128, blocks_per_sm=2, policy=8, contiguous=0, reverse=1, keep_mib=0),
+    # the rolling-slot Dot kernel (the elementwise kernels ignore `pipeline`)
+    dict(kind=0, vec_bytes=32, unroll=2, threads=512, blocks_per_sm=0, policy=4, contiguous=0, pipeline=1),
+    dict(kind=0, vec_bytes=32, unroll=4, threads=256, blocks_per_sm=1, policy=0, contiguous=0, pipeline=1),
+    dict(kind=0, vec_bytes=32, unroll=2, threads=128, blocks_per_sm=3, policy=4, contiguous=0, pipeline=1, two_pass=1),
 ]
 BULK_TUNINGS = [
     dict(kind=1, threads=128, blocks_per_sm=1, chunk_bytes=1024, stages=2),

@@ -204,8 +204,10 @@ def test_dot_matches_the_compensated_oracle(so, torch, oracle, t, tuning):
 
 
 @pytest.mark.parametrize("t", ["f64", "f32"])
-@pytest.mark.parametrize("tuning", [dict(), dict(kind=0, vec_bytes=16, unroll=4, threads=128, blocks_per_sm=1), dict(kind=1)],
-                         ids=["default", "vec16", "bulk"])
+@pytest.mark.parametrize("tuning", [dict(), dict(kind=0, vec_bytes=16, unroll=4, threads=128, blocks_per_sm=1), dict(kind=1),
+                                    dict(kind=0, pipeline=0, unroll=4, blocks_per_sm=0), dict(kind=0, pipeline=1, unroll=2, blocks_per_sm=0),
+                                    dict(kind=0, pipeline=1, unroll=4, threads=256, blocks_per_sm=3)],
+                         ids=["default", "vec16", "bulk", "tiles", "roll2", "roll4"])
 def test_dot_visits_every_index_exactly_once(so, torch, oracle, t, tuning):
     """dot(x, e_k) = x_k exactly, for k in the tail, at tile and block boundaries: no index is
     skipped and none is counted twice (dot(x, 1) on integers would double-count otherwise)."""
