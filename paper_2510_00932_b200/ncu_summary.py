@@ -26,7 +26,7 @@ OP_OF_CODE = {0: "copy", 1: "scale", 2: "add", 3: "triad"}
 
 
 def op_of_kernel(name: str):
-    if "dot_pass1_kernel" in name or "dot_comp_kernel" in name:
+    if "dot_pass1_kernel" in name or "dot_roll_kernel" in name or "dot_comp_kernel" in name:
         return "dot"
     m = re.search(r"ew_vec_kernel<[^,]+,\s*(?:\(int\))?(\d)", name)
     return OP_OF_CODE.get(int(m.group(1))) if m else None

@@ -63,7 +63,9 @@ def run_shapes(sizes=((1 << 25), (1 << 28)), iters=20, dtype="f64"):
     threads per block x vectors in flight per thread x grid form x cache-hint set, each timed
     op-major (`iters` launches in a row, one CUDA-event pair) on uniform [0,1) arrays, plus the
     time of one chain step (copy, scale, add, triad, dot) with the elementwise kernels or Dot set to
-    that shape and everything else at its default. This is the sweep the defaults are chosen from."""
+    that shape and everything else at its default. This is the sweep the defaults are chosen from.
+    (Op-major launches do not consume their predecessor's output, so policies 7 and 8 store
+    evict-first there, like 4; their two-phase stores show in the chain column.)"""
     import itertools
     import torch
     from . import harness, inputs
@@ -76,8 +78,9 @@ def run_shapes(sizes=((1 << 25), (1 << 28)), iters=20, dtype="f64"):
     stream = torch.cuda.current_stream()
     ew_shapes = [dict(threads=th, unroll=u, blocks_per_sm=bps, policy=pol)
                  for th, u, bps, pol in itertools.product((128, 256, 512), (1, 2, 4), (0, 4, 8), (4, 5, 7))]
-    dot_shapes = [dict(threads=th, unroll=u, blocks_per_sm=bps, policy=pol)
-                  for th, u, bps, pol in itertools.product((256, 512), (1, 2, 4), (0, 1, 2, 3, 4), (0, 4))]
+    dot_shapes = [dict(threads=th, unroll=u, blocks_per_sm=bps, policy=pol, pipeline=pipe)
+                  for pipe, th, u, bps, pol in itertools.product((0, 1), (256, 512), (1, 2, 4), (0, 1, 2, 3, 4), (0, 4))
+                  if not (pipe == 1 and u == 1)]
     rows = []
     for n in sizes:
         w = inputs.sweep_workload(dtype, n)
@@ -130,14 +133,15 @@ def shapes_markdown(rows) -> str:
         out.append(f"### n = {n} (fp64, {n * 8 / 2**20:.0f} MiB per array); microseconds per launch, op-major; chain = one step of the five kernels\n")
         out.append("default tuning: " + ", ".join(f"{op} {base[op]}" for op in ("copy", "scale", "add", "triad", "dot")) + f", chain {base['chain_us']}\n")
         for group, ops in (("ew", ("copy", "scale", "add", "triad")), ("dot", ("dot",))):
-            out.append("| threads | unroll | grid | policy | " + " | ".join(ops) + " | chain step |")
-            out.append("|---|---|---|---|" + "---|" * (len(ops) + 1))
+            out.append(("| kernel " if group == "dot" else "") + "| threads | unroll | grid | policy | " + " | ".join(ops) + " | chain step |")
+            out.append(("|---" if group == "dot" else "") + "|---|---|---|---|" + "---|" * (len(ops) + 1))
             for r in mine[1:]:
                 sh = r["shape"]
                 if sh["group"] != group:
                     continue
                 grid = "block per tile" if sh["blocks_per_sm"] == 0 and group == "ew" else ("automatic" if sh["blocks_per_sm"] == 0 else f"{sh['blocks_per_sm']} per SM")
-                out.append(f"| {sh['threads']} | {sh['unroll']} | {grid} | {sh['policy']} | " + " | ".join(f"{r[o]:.1f}" for o in ops) + f" | {r['chain_us']:.1f} |")
+                kern = ("| rolling slots " if sh.get("pipeline") else "| tiles ") if group == "dot" else ""
+                out.append(kern + f"| {sh['threads']} | {sh['unroll']} | {grid} | {sh['policy']} | " + " | ".join(f"{r[o]:.1f}" for o in ops) + f" | {r['chain_us']:.1f} |")
             out.append("")
     return "\n".join(out) + "\n"
 
