@@ -186,6 +186,34 @@ def check_parity(oracle, w, seeded, device_arrays, device_dot, steps, nthreads):
             "dot_condition_number": mags / abs(d) if d != 0 else None}
 
 
+def host_link_ceiling(torch, device, nbytes: int, reps: int = 5):
+    """What the host link itself delivers for pinned memory, to hold the end-to-end figure against:
+    GB/s of a host-to-device copy alone, of a device-to-host copy alone, and per direction when one of
+    each run at the same time on two streams (plain cudaMemcpyAsync through torch; no kernel involved)."""
+    n = nbytes // 8
+    h_in, h_out = torch.empty(n, dtype=torch.float64).pin_memory(), torch.empty(n, dtype=torch.float64).pin_memory()
+    d_in, d_out = torch.empty(n, dtype=torch.float64, device=device), torch.zeros(n, dtype=torch.float64, device=device)
+    s_up, s_down = torch.cuda.Stream(device), torch.cuda.Stream(device)
+
+    def timed(up: bool, down: bool):
+        best = float("inf")
+        for _ in range(reps):
+            torch.cuda.synchronize(device)
+            t0 = time.perf_counter()
+            if up:
+                with torch.cuda.stream(s_up):
+                    d_in.copy_(h_in, non_blocking=True)
+            if down:
+                with torch.cuda.stream(s_down):
+                    h_out.copy_(d_out, non_blocking=True)
+            torch.cuda.synchronize(device)
+            best = min(best, time.perf_counter() - t0)
+        return nbytes / best / 1e9
+
+    return {"h2d_alone_gbs": round(timed(True, False), 1), "d2h_alone_gbs": round(timed(False, True), 1),
+            "each_way_when_both_run_gbs": round(timed(True, True), 1), "bytes_per_copy": nbytes}
+
+
 def versions(torch):
     import subprocess
     import numpy as np
@@ -329,7 +357,7 @@ def run_ours(args):
     # end to end: host buffers in, host buffers out, through the library's host entry point
     ha, hb, hc = (p.numpy() for p in pinned)              # the pinned arrays are updated in place from here on
     e2e_steps = args.e2e_steps if chain_cap is None else min(args.e2e_steps, 8)
-    e2e_value, e2e_dot = None, None                       # --e2e-steps 0 (profiling runs) skips this leg
+    e2e_value, e2e_dot, e2e_link = None, None, None       # --e2e-steps 0 (profiling runs) skips this leg
     if e2e_steps > 0:
         warm_e2e = [v[:1 << 22].copy() for v in (ha, hb, hc)]
         so.chain_host(*warm_e2e, w.scalar)                # creates the library's device ring; leaves the arrays alone
@@ -340,6 +368,11 @@ def run_ours(args):
         torch.cuda.synchronize(device)
         e2e_ms = (time.perf_counter() - t0) * 1e3
         e2e_value, _ = harness.whole_job_gbs(harness.step_bytes(n, itemsize) * e2e_steps, e2e_ms, device)
+        if rank == 0 and world == 1:
+            # the link's own ceiling: a step moves 3 arrays each way, so at best it takes 3nB / (GB/s each way)
+            e2e_link = host_link_ceiling(torch, device, 3 * n * itemsize)
+            ceiling = harness.step_bytes(n, itemsize) / (3 * n * itemsize / e2e_link["each_way_when_both_run_gbs"])
+            e2e_link.update({"e2e_ceiling_gbs": round(ceiling, 1), "e2e_frac_of_ceiling": round(e2e_value / ceiling, 4)})
 
     peak, peak_src = harness.measured_peak()
     extra = {}
@@ -421,7 +454,7 @@ def run_ours(args):
             "clocks": clocks, "parity": parity, "per_op_isolated": per_op_isolated, "per_op": per_op, "roofline": roofline,
             "cpu_baseline": cpu_baseline,
             "e2e": {"value": None if e2e_value is None else round(e2e_value, 2), "unit": UNIT, "h2d_bytes_per_step": 3 * n * itemsize,
-                    "d2h_bytes_per_step": 3 * n * itemsize + itemsize, "steps": e2e_steps},
+                    "d2h_bytes_per_step": 3 * n * itemsize + itemsize, "steps": e2e_steps, "host_link": e2e_link},
             "gpu_launches": int(launches), "gpu_launches_all_regions": int(launches_all),
             "frac_nominal_8tbs": round(value / world / harness.NOMINAL_HBM_GBS, 4),
             "other_workloads": extra, "shmem_mix": shmem, "versions": versions(torch), "tuning": sig,
