@@ -12,7 +12,8 @@
 //
 // A block stages a tile in shared memory; thread t owns VW adjacent columns, i.e. one 4*VW-byte
 // piece of every row, eight pieces in all. A round is eight shared-memory loads, one three-input
-// add per word, and eight shared-memory stores per thread; every value travels through shared memory every round
+// add per word, and eight shared-memory stores per thread (the store of row k is issued as soon as
+// row k + 2 has been loaded, so loads and stores alternate); every value travels through shared memory every round
 // (the accesses are inline PTX, so the compiler cannot keep them in registers across rounds).
 // Pieces of one row are contiguous across the threads of a warp: no bank conflicts at any width.
 // No thread ever reads a column another thread writes, so there is no barrier in the loop --
@@ -84,18 +85,22 @@ shmem_mix_kernel(const uint32_t *x, uint32_t *out, unsigned rounds, size_t n) {
 #pragma unroll
         for (int k = 0; k < kRows; ++k) sts<VW>(mine + k * kRowBytes, row[k]);
         for (unsigned r = 0; r < rounds; ++r) {
-#pragma unroll
-            for (int k = 0; k < kRows; ++k) lds<VW>(row[k], mine + k * kRowBytes);
+            // Row k's new value needs the old rows k, k + 1 and k + 2 only, so its store is issued as soon as
+            // row k + 2 has been loaded: loads and stores alternate instead of eight of one kind following
+            // eight of the other, and a warp's round is not one long load-then-store dependence.
+            lds<VW>(row[0], mine);
+            lds<VW>(row[1], mine + kRowBytes);
             const Piece<VW> first = row[0], second = row[1];
 #pragma unroll
-            for (int k = 0; k < kRows; ++k) {           // ascending k: rows k + 1 and k + 2 still hold old values
+            for (int k = 0; k < kRows; ++k) {
+                if (k + 2 < kRows) lds<VW>(row[k + 2], mine + (k + 2) * kRowBytes);
+                Piece<VW> nv;
 #pragma unroll
                 for (int e = 0; e < VW; ++e)
-                    row[k].w[e] += (k + 1 < kRows ? row[k + 1].w[e] : first.w[e]) +
-                                   (k + 2 < kRows ? row[k + 2].w[e] : (k + 2 == kRows ? first.w[e] : second.w[e]));
+                    nv.w[e] = row[k].w[e] + (k + 1 < kRows ? row[k + 1].w[e] : first.w[e]) +
+                              (k + 2 < kRows ? row[k + 2].w[e] : (k + 2 == kRows ? first.w[e] : second.w[e]));
+                sts<VW>(mine + k * kRowBytes, nv);
             }
-#pragma unroll
-            for (int k = 0; k < kRows; ++k) sts<VW>(mine + k * kRowBytes, row[k]);
         }
 #pragma unroll
         for (int k = 0; k < kRows; ++k) lds<VW>(row[k], mine + k * kRowBytes);
