@@ -30,7 +30,10 @@ PAPER_NUM_TIMES = (100, 200, 300)
 class ChainGraph:
     """The five-kernel pass over (a, b, c), captured once and replayed with one launch per
     iteration. The Dot's output pointer is pinned host memory (device-accessible under unified
-    addressing), so the result lands on the host without a copy node in the graph."""
+    addressing), so the result lands on the host without a copy node in the graph. The captured Dot
+    uses one of the library's workspace slots reserved for graphs (never handed to ordinary calls),
+    and the elementwise launches keep the traversal directions chosen at capture time; both are part
+    of the graph. Replays of one ChainGraph must not overlap each other (they share that slot)."""
 
     def __init__(self, a, b, c, scalar: float):
         import torch

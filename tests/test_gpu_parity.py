@@ -230,6 +230,30 @@ def test_dot_visits_every_index_exactly_once(so, torch, oracle, t, tuning):
     assert out.item() == float(_npdt(t)(n))
 
 
+@pytest.mark.parametrize("t", ["f64", "f32"])
+@pytest.mark.parametrize("shape", [dict(unroll=2, threads=512, blocks_per_sm=0), dict(unroll=4, threads=256, blocks_per_sm=1),
+                                   dict(unroll=2, threads=128, blocks_per_sm=2)], ids=["2x512", "4x256", "2x128"])
+def test_rolling_slot_dot_counts_every_element_around_its_round_boundaries(so, torch, t, shape):
+    """dot(1, 1) = n exactly (every partial sum is an integer below 2^53) for n just below, on and just
+    above a tile, one pass of all blocks, one round of all slots and two rounds, plus a ragged end: a
+    slot that skipped its last reload, or a tile counted by two slots, changes the count."""
+    so.set_tuning("dot", t, pipeline=1, vec_bytes=32, kind=0, **shape)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    epv = 4 if t == "f64" else 8
+    tile = shape["threads"] * epv
+    grid = (shape["blocks_per_sm"] or 2) * sms
+    marks = [tile, grid * tile, shape["unroll"] * grid * tile, 2 * shape["unroll"] * grid * tile]
+    sizes = sorted({m + d for m in marks for d in (-tile - 1, -1, 0, 1, epv, tile - 1, tile + 3)} | {1, 5, epv, 3 * marks[2] + 2 * tile + 7})
+    biggest = max(sizes)
+    ones = torch.ones(biggest, dtype=torch.float64 if t == "f64" else torch.float32, device="cuda")
+    out = torch.zeros(1, dtype=ones.dtype, device="cuda")
+    for n in sizes:
+        if n <= 0 or (t == "f32" and n > (1 << 24)):        # float holds integers exactly only up to 2^24
+            continue
+        so.dot(ones[:n], ones[:n], out)
+        assert out.item() == float(n), f"n={n}"
+
+
 def test_dot_f32_output_is_rounded_to_float(so, torch):
     n = (1 << 24) + 7
     ones = torch.ones(n, dtype=torch.float32, device="cuda")
