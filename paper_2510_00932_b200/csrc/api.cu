@@ -408,8 +408,8 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
             return STREAMOPS_ERR_WORKSPACE;
         }
         // pieces of equal length (the last one shorter), at most kChainMaxPieces of them. (Shorter first
-        // and last pieces were measured and change nothing: the time lost against the link's own rate
-        // is spent in the hand-overs between the three streams, not in filling and draining the pipeline.)
+        // and last pieces were measured and change nothing: filling and draining the pipeline is not where
+        // the time against the link's own rate goes.)
         size_t piece = g_chain_piece_bytes.load() / sizeof(T);
         while ((n + piece - 1) / piece > kChainMaxPieces) piece *= 2;
         const size_t pieces = n ? (n + piece - 1) / piece : 0;
