@@ -1,10 +1,10 @@
 """Turns an ncu launch list with DRAM counters into the per-kernel traffic summary bench.py reads.
 
-    ncu --cache-control none --clock-control none --csv --log-file gpurun_out/opmajor_dram.csv \
+    ncu --cache-control none --clock-control none --csv --log-file opmajor_dram.csv \
         --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum \
         -k regex:"ew_vec_kernel|dot_pass1" -c 200 \
         python bench.py --steps 3 --warmup 3 --cpu-seconds 0 --e2e-steps 0 --no-shmem --no-parity --extra ""
-    python -m paper_2510_00932_b200.ncu_summary gpurun_out/opmajor_dram.csv --workload c2 \
+    python -m paper_2510_00932_b200.ncu_summary opmajor_dram.csv --workload c2 \
         --command "<the ncu command above>"
 
 bench.py's op-major region launches each kernel several times in a row; in the launch list that is a
