@@ -256,6 +256,21 @@ int streamops_check(streamops_stream_t stream);
  * output of such a launch is incomplete. Nothing faults and nothing waits without bound. */
 int streamops_set_wait_limit(unsigned tries);
 
+/* Index checking (debugging builds only: the library built with -DSTREAMOPS_CHECK_INDICES, which
+ * `python -m paper_2510_00932_b200.build --checked` writes to libstreamops_checked.so). In such a build every
+ * global-memory access of the register-vector elementwise and Dot kernels is first checked against the
+ * length of its array; an access that does not fit is not made, and the first one is recorded.
+ * streamops_index_violation synchronises the device and returns 1 if an access was refused since the last
+ * call (filling in which access -- 1/2/3 elementwise load of x / load of y / store, 4 elementwise ragged end,
+ * 5/6/7 the same for Dot, 99 the self-test --, its byte offset and the array's byte length, and clearing
+ * the record), 0 if none was, and a negative value in a build without checking (-STREAMOPS_ERR_ARG) or on a
+ * CUDA error. streamops_index_selftest launches a kernel that only ASKS the checker about an access of
+ * `width` bytes at byte `offset` of an array of `limit` bytes, and about the last access that fits, without
+ * touching memory: it returns bit 0 = the first was accepted, bit 1 = the second was (so 2 for an `offset`
+ * that does not fit, after which streamops_index_violation reports where = 99), negative as above. */
+int streamops_index_violation(int *where, unsigned long long *offset, unsigned long long *limit);
+int streamops_index_selftest(unsigned long long offset, unsigned long long width, unsigned long long limit);
+
 const char *streamops_status_string(int status);
 int streamops_last_cuda_error(void); /* the cudaError_t behind the last STREAMOPS_ERR_CUDA */
 

@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "../../include/streamops.h"
+#include "indexcheck.cuh"
 #include "internal.cuh"
 
 using namespace streamops;
@@ -475,9 +476,27 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
 }  // namespace
 
 namespace streamops {
+// Readers of the per-translation-unit index-violation records (checking builds register one per
+// kernel file during static initialisation; an ordinary build registers none).
+namespace {
+constexpr int kMaxViolationReaders = 16;
+violation_reader_t g_violation_readers[kMaxViolationReaders];
+int g_violation_reader_count = 0;
+}  // namespace
+void register_violation_reader(violation_reader_t reader) {
+    if (g_violation_reader_count < kMaxViolationReaders) g_violation_readers[g_violation_reader_count++] = reader;
+}
 int note_cuda_error(cudaError_t e) { return cuda_fail(e); }
 void note_launches(int n) { g_launches.fetch_add((unsigned long long)n); }
 }  // namespace streamops
+
+#ifdef STREAMOPS_CHECK_INDICES
+// Asks index_ok about an access that does not fit, without making any access: exercises the record.
+__global__ void index_selftest_kernel(unsigned long long offset, unsigned long long width, unsigned long long limit, int *verdicts) {
+    verdicts[0] = index_ok((size_t)offset, (size_t)width, (size_t)limit, W_SELFTEST) ? 1 : 0;
+    verdicts[1] = index_ok((size_t)(limit - width), (size_t)width, (size_t)limit, W_SELFTEST) ? 1 : 0;
+}
+#endif
 
 extern "C" {
 
@@ -655,6 +674,44 @@ const char *streamops_status_string(int status) {
 int streamops_set_wait_limit(unsigned tries) {
     g_wait_limit.store(tries == 0 ? (1u << 22) : tries);
     return STREAMOPS_OK;
+}
+
+int streamops_index_violation(int *where, unsigned long long *offset, unsigned long long *limit) {
+#ifdef STREAMOPS_CHECK_INDICES
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return -cuda_fail(e);
+    for (int i = 0; i < g_violation_reader_count; ++i) {
+        IndexViolation v{0, 0, 0, 0};
+        if ((e = g_violation_readers[i](&v, true)) != cudaSuccess) return -cuda_fail(e);
+        if (v.flag) {
+            if (where) *where = v.where;
+            if (offset) *offset = v.offset;
+            if (limit) *limit = v.limit;
+            return 1;
+        }
+    }
+    return 0;
+#else
+    (void)where; (void)offset; (void)limit;
+    return -STREAMOPS_ERR_ARG;            // not a checking build
+#endif
+}
+
+int streamops_index_selftest(unsigned long long offset, unsigned long long width, unsigned long long limit) {
+#ifdef STREAMOPS_CHECK_INDICES
+    if (width == 0 || width > limit) return -STREAMOPS_ERR_ARG;
+    int *verdicts = nullptr;
+    if (cudaMalloc(&verdicts, 2 * sizeof(int)) != cudaSuccess) { (void)cudaGetLastError(); return -STREAMOPS_ERR_WORKSPACE; }
+    index_selftest_kernel<<<1, 1>>>(offset, width, limit, verdicts);
+    int host[2] = {-1, -1};
+    cudaError_t e = cudaMemcpy(host, verdicts, sizeof host, cudaMemcpyDeviceToHost);
+    cudaFree(verdicts);
+    if (e != cudaSuccess) return -cuda_fail(e);
+    return host[0] | (host[1] << 1);       // bit 0: the probed access was accepted; bit 1: the last fitting access was
+#else
+    (void)offset; (void)width; (void)limit;
+    return -STREAMOPS_ERR_ARG;
+#endif
 }
 
 int streamops_last_cuda_error(void) { return g_last_cuda_error.load(); }

@@ -17,6 +17,7 @@
 // by whichever block arrives last at an atomic ticket: the ticket only elects WHO does pass 2,
 // the order of the additions is by block index, so the bits of the result never depend on
 // block scheduling, on the stream, or on what else the GPU is running.
+#include "indexcheck.cuh"
 #include "internal.cuh"
 #include "memops.cuh"
 #include "reduce.cuh"
@@ -57,9 +58,21 @@ dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned lo
         const size_t v0 = (reverse ? ntiles - 1 - tile : tile) * tile_vecs + threadIdx.x;
         Vec<VB> xv[U], yv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+        for (int u = 0; u < U; ++u) {
+#ifdef STREAMOPS_CHECK_INDICES
+            xv[u] = Vec<VB>{};                         // an access a checking build refuses contributes zero
+#endif
+            if (index_ok((v0 + (size_t)u * blockDim.x) * VB, VB, n * sizeof(T), W_DOT_LOAD_X))
+                ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+        }
 #pragma unroll
-        for (int u = 0; u < U; ++u) ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+        for (int u = 0; u < U; ++u) {
+#ifdef STREAMOPS_CHECK_INDICES
+            yv[u] = Vec<VB>{};
+#endif
+            if (index_ok((v0 + (size_t)u * blockDim.x) * VB, VB, n * sizeof(T), W_DOT_LOAD_Y))
+                ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2pol);
+        }
 #pragma unroll
         for (int u = 0; u < U; ++u) acc[u] = fold_vec<T, VB>(acc[u], xv[u], yv[u]);
     }
@@ -110,7 +123,7 @@ dot_roll_kernel(const T *x, const T *y, size_t n, double *partials, unsigned lon
 #pragma unroll
     for (int s = 0; s < S; ++s) {
         const size_t o = off + (size_t)s * slot_stride;
-        if (o < end) {
+        if (o < end && index_ok(o, VB, n * sizeof(T), W_DOT_LOAD_X)) {
             ldg<POL>(xv[s], xb + o, l2pol);
             ldg<POL>(yv[s], yb + o, l2pol);
         }
@@ -122,7 +135,7 @@ dot_roll_kernel(const T *x, const T *y, size_t n, double *partials, unsigned lon
             if (o < end) {
                 acc[s] = fold_vec<T, VB>(acc[s], xv[s], yv[s]);
                 const size_t next = o + round_stride;
-                if (next < end) {
+                if (next < end && index_ok(next, VB, n * sizeof(T), W_DOT_LOAD_X)) {
                     ldg<POL>(xv[s], xb + next, l2pol);
                     ldg<POL>(yv[s], yb + next, l2pol);
                 }

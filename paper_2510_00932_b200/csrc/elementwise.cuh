@@ -14,6 +14,7 @@
 // Arithmetic uses the explicit round-to-nearest intrinsics (__dmul_rn, __dadd_rn, __fmul_rn,
 // __fadd_rn), which the compiler never contracts into a fused multiply-add.
 #pragma once
+#include "indexcheck.cuh"
 #include "internal.cuh"
 #include "memops.cuh"
 
@@ -59,6 +60,7 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int
     const size_t nvec = n / EPV;
     const size_t tile_vecs = (size_t)blockDim.x * U;
     const size_t ntiles = nvec / tile_vecs;          // full tiles only
+    const size_t nbytes = n * sizeof(T);             // what index_ok checks against (checking builds only)
     size_t tile, end, step;
     if (contiguous) {
         const size_t per = (ntiles + gridDim.x - 1) / gridDim.x;
@@ -74,32 +76,41 @@ ew_vec_kernel(const T *x, const T *y, T *out, T s, size_t n, int contiguous, int
         const uint64_t stpol = (POL == 8 && tile >= hot_tiles) ? l2.st_late : l2.st;
         Vec<VB> xv[U], yv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
+        for (int u = 0; u < U; ++u)
+            if (index_ok((v0 + (size_t)u * blockDim.x) * VB, VB, nbytes, W_EW_LOAD_X))
+                ldg<POL>(xv[u], xb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
         if constexpr (kUsesY<OP>) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
+            for (int u = 0; u < U; ++u)
+                if (index_ok((v0 + (size_t)u * blockDim.x) * VB, VB, nbytes, W_EW_LOAD_Y))
+                    ldg<POL>(yv[u], yb + (v0 + (size_t)u * blockDim.x) * VB, l2.ld);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) apply_vec<T, OP, VB>(xv[u], yv[u], s);
         if (POL == 7 && tile >= hot_tiles) {       // second phase of policy 7: plain stores (uniform per tile)
 #pragma unroll
-            for (int u = 0; u < U; ++u) stg<0>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], 0);
+            for (int u = 0; u < U; ++u)
+                if (index_ok((v0 + (size_t)u * blockDim.x) * VB, VB, nbytes, W_EW_STORE))
+                    stg<0>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], 0);
         } else {
 #pragma unroll
-            for (int u = 0; u < U; ++u) stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], stpol);
+            for (int u = 0; u < U; ++u)
+                if (index_ok((v0 + (size_t)u * blockDim.x) * VB, VB, nbytes, W_EW_STORE))
+                    stg<POL>(ob + (v0 + (size_t)u * blockDim.x) * VB, xv[u], stpol);
         }
     }
     // ragged end, by the block that is next in line for a tile
     if (blockIdx.x == (unsigned)(ntiles % gridDim.x)) {
         for (size_t v = ntiles * tile_vecs + threadIdx.x; v < nvec; v += blockDim.x) {
             Vec<VB> xv, yv;
+            if (!index_ok(v * VB, VB, nbytes, W_EW_TAIL)) continue;
             ldg<0>(xv, xb + v * VB, 0);
             if constexpr (kUsesY<OP>) ldg<0>(yv, yb + v * VB, 0);
             apply_vec<T, OP, VB>(xv, yv, s);
             stg<0>(ob + v * VB, xv, 0);
         }
         const size_t i = nvec * EPV + threadIdx.x;   // fewer than EPV elements remain
-        if (i < n) {
+        if (i < n && index_ok(i * sizeof(T), sizeof(T), nbytes, W_EW_TAIL)) {
             if constexpr (OP == OP_COPY) out[i] = x[i];
             else out[i] = apply<T, OP>(x[i], kUsesY<OP> ? y[i] : T(0), s);
         }

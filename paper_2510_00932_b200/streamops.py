@@ -12,7 +12,9 @@ import os
 from dataclasses import dataclass
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libstreamops.so")
+# STREAMOPS_LIBRARY selects another build of the same library, e.g. the index-checking one
+# (libstreamops_checked.so, written by `python -m paper_2510_00932_b200.build --checked`)
+LIB_PATH = os.environ.get("STREAMOPS_LIBRARY") or os.path.join(_HERE, "libstreamops.so")
 
 OPS = ("copy", "scale", "add", "triad", "dot")
 OP_CODE = {name: i for i, name in enumerate(OPS)}
@@ -77,6 +79,9 @@ def lib() -> ctypes.CDLL:
         L.streamops_policy_name.argtypes, L.streamops_policy_name.restype = [ci], ctypes.c_char_p
         L.streamops_check.argtypes, L.streamops_check.restype = [vp], ci
         L.streamops_set_wait_limit.argtypes, L.streamops_set_wait_limit.restype = [ctypes.c_uint], ci
+        ullp = ctypes.POINTER(ctypes.c_ulonglong)
+        L.streamops_index_violation.argtypes, L.streamops_index_violation.restype = [ctypes.POINTER(ci), ullp, ullp], ci
+        L.streamops_index_selftest.argtypes, L.streamops_index_selftest.restype = [ctypes.c_ulonglong] * 3, ci
         L.streamops_status_string.argtypes, L.streamops_status_string.restype = [ci], ctypes.c_char_p
         L.streamops_last_cuda_error.argtypes, L.streamops_last_cuda_error.restype = [], ci
         L.streamops_launch_count.argtypes, L.streamops_launch_count.restype = [], ctypes.c_ulonglong
@@ -322,6 +327,23 @@ def check(stream=None):
 def set_wait_limit(tries: int):
     """Attempts a wait inside the bulk-copy pipelines makes before giving up (0 = default)."""
     _raise(lib().streamops_set_wait_limit(int(tries)))
+
+
+def index_violation():
+    """Index-checking builds: None if no access was refused since the last call, else a dict with the
+    kind of access, its byte offset and the array's byte length. Raises in an ordinary build."""
+    where, off, lim = ctypes.c_int(0), ctypes.c_ulonglong(0), ctypes.c_ulonglong(0)
+    rc = lib().streamops_index_violation(ctypes.byref(where), ctypes.byref(off), ctypes.byref(lim))
+    if rc < 0:
+        _raise(-rc)
+    return None if rc == 0 else {"where": where.value, "offset": off.value, "limit": lim.value}
+
+
+def index_selftest(offset: int, width: int, limit: int) -> int:
+    rc = lib().streamops_index_selftest(int(offset), int(width), int(limit))
+    if rc < 0:
+        _raise(-rc)
+    return rc
 
 
 def launch_count() -> int:
