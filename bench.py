@@ -226,7 +226,7 @@ def versions(torch):
             "driver_and_gpu": drv, "python": sys.version.split()[0]}
 
 
-def run_extra(torch, so, harness, inputs, name, K, device, stream, peak):
+def run_extra(torch, so, harness, inputs, name, K, device, stream, peak, pin_gbs=None):
     """Op-major timing of another named workload (few launches), so that the record carries the
     single-precision and the 2 GiB-per-array figures beside the headline one."""
     w = inputs.WORKLOADS[name]
@@ -237,7 +237,7 @@ def run_extra(torch, so, harness, inputs, name, K, device, stream, peak):
     dd = torch.zeros(1, dtype=da.dtype, device=device)
     ms = time_op_major(torch, make_calls(so, w, da, db, dc, dd), K, device, stream, harness)
     so.check()
-    rep = harness.per_op_report(ms, w.n, w.itemsize, peak)
+    rep = harness.per_op_report(ms, w.n, w.itemsize, peak, pin_gbs)
     return {"dtype": w.dtype, "n": w.n, "dist": w.dist, "launches_per_op": K, "order": "op-major", "per_op_isolated": rep}
 
 
@@ -375,12 +375,17 @@ def run_ours(args):
             e2e_link.update({"e2e_ceiling_gbs": round(ceiling, 1), "e2e_frac_of_ceiling": round(e2e_value / ceiling, 4)})
 
     peak, peak_src = harness.measured_peak()
+    # what the memory pins could carry: data rate x bus width, both read from the device at run time
+    props = torch.cuda.get_device_properties(device)
+    pin_gbs = None
+    if getattr(props, "memory_clock_rate", 0) and getattr(props, "memory_bus_width", 0):
+        pin_gbs = harness.pin_bandwidth_gbs(props.memory_clock_rate, props.memory_bus_width)
     extra = {}
     if rank == 0 and world == 1:
         del calls, da, db, dc
         torch.cuda.empty_cache()
         for name in [x for x in args.extra.split(",") if x and x != w.name]:
-            extra[name] = run_extra(torch, so, harness, inputs, name, max(5, min(K, 20)), device, stream, peak)
+            extra[name] = run_extra(torch, so, harness, inputs, name, max(5, min(K, 20)), device, stream, peak, pin_gbs)
             torch.cuda.empty_cache()
 
     # the shared-memory exchange microkernel, at the paper's default repetition count (own line, not part of `value`)
@@ -405,10 +410,10 @@ def run_ours(args):
                                      "cores": nthreads, "kind": "oracle",
                                      "sample": "one all-threads pass over n=2^22 words, 600 rounds, same byte accounting"}
 
-    per_op = harness.per_op_report(op_ms, n, itemsize, peak)
+    per_op = harness.per_op_report(op_ms, n, itemsize, peak, pin_gbs)
     for name in per_op:
         per_op[name]["best_gbs"] = round(harness.op_bytes(name, n, itemsize) / (op_ms_best[name] * 1e-3) / 1e9, 1)
-    per_op_isolated = harness.per_op_report(iso_ms, n, itemsize, peak)
+    per_op_isolated = harness.per_op_report(iso_ms, n, itemsize, peak, pin_gbs)
     # the kernel that takes the largest share of the op-major time is the one the roofline entry describes
     dominant = max(iso_ms, key=lambda k: iso_ms[k])
     sig = tuning_signature(so, w.dtype)
@@ -417,6 +422,10 @@ def run_ours(args):
                 "peak_source": f"of {peak_src}", "unit": "GB/s",
                 "frac": round(per_op_isolated[dominant]["gbs"] / peak, 4),
                 "frac_nominal_8tbs": per_op_isolated[dominant]["frac_nominal_8tbs"], "traffic": traffic,
+                "pin_bandwidth_gbs": None if pin_gbs is None else round(pin_gbs, 1),
+                "pin_bandwidth_source": "2 x memory clock x bus width as the device reports them "
+                                        f"({props.memory_clock_rate / 1e3:.0f} MHz, {props.memory_bus_width} bits)",
+                "frac_of_pin_bandwidth": None if pin_gbs is None else round(per_op_isolated[dominant]["gbs"] / pin_gbs, 4),
                 "region": "op-major: the kernel launched K times in a row, one CUDA-event pair around the K; "
                           "no cached lines inherited from other kernels. The peak is a plain 1:1 copy; a 2:1 read-heavy "
                           "kernel can read a little above it"}

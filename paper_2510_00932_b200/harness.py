@@ -143,13 +143,22 @@ def summarize_clock_lines(lines) -> dict:
             "samples": len(sm)}
 
 
-def per_op_report(durations_ms: dict, n: int, itemsize: int, peak_gbs: float) -> dict:
-    """GB/s per operation from average launch durations, with both roofline fractions."""
+def pin_bandwidth_gbs(memory_clock_khz: float, bus_width_bits: int) -> float:
+    """What the memory pins of the device can carry: double data rate x bus width, from the two
+    attributes the device reports (a B200 with 7680 of 8192 bits enabled at 3996 MHz: 7672 GB/s)."""
+    return 2.0 * memory_clock_khz * 1e3 * bus_width_bits / 8 / 1e9
+
+
+def per_op_report(durations_ms: dict, n: int, itemsize: int, peak_gbs: float, pin_gbs: float | None = None) -> dict:
+    """GB/s per operation from average launch durations, with the roofline fractions: of the measured
+    copy rate, of the nominal 8 TB/s, and (when given) of the device's own pin bandwidth."""
     out = {}
     for op, ms in durations_ms.items():
         gbs = op_bytes(op, n, itemsize) / (ms * 1e-3) / 1e9
         out[op] = {"ms": round(ms, 5), "gbs": round(gbs, 1), "frac_measured_peak": round(gbs / peak_gbs, 4),
                    "frac_nominal_8tbs": round(gbs / NOMINAL_HBM_GBS, 4)}
+        if pin_gbs:
+            out[op]["frac_pin_bandwidth"] = round(gbs / pin_gbs, 4)
     return out
 
 

@@ -172,3 +172,10 @@ def test_traffic_summary_round_trip(tmp_path, monkeypatch):
     assert harness.captured_traffic("c2", "add", t) == 536_950_000 + 268_400_000
     assert harness.captured_traffic("c2", "add", dict(t, unroll=4)) is None
     assert harness.captured_traffic("c2", "dot", so.get_tuning("dot", "f64").as_dict()) is None
+
+
+def test_pin_bandwidth_from_device_attributes():
+    assert harness.pin_bandwidth_gbs(3996000, 7680) == pytest.approx(7672.3, abs=0.1)
+    assert harness.pin_bandwidth_gbs(3996000, 8192) == pytest.approx(8183.8, abs=0.1)
+    rep = harness.per_op_report({"dot": 0.0731}, 1 << 25, 8, 6548.8, 7672.3)
+    assert rep["dot"]["frac_pin_bandwidth"] == pytest.approx(536870912 / 0.0731e-3 / 1e9 / 7672.3, abs=1e-3)
