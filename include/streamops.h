@@ -149,8 +149,10 @@ int streamops_chain_f64(double *a, double *b, double *c, double *dot_out, double
 int streamops_chain_f32(float *a, float *b, float *c, float *dot_out, double scalar, size_t n, streamops_stream_t stream);
 
 /* One pass of the five kernels over three HOST arrays of n elements each, in the textbook
- * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). The arrays are cut into pieces
- * of 16 MiB per array; each piece is copied into a ring of four device stages (three piece buffers
+ * STREAM dataflow: c <- a; b <- s*c; c <- a+b; a <- b+s*c; dot(a, b). On return a, b and c hold the results;
+ * of their contents on entry only a's are read (the dataflow overwrites c and b before reading them, so b and c
+ * are outputs only and are not copied to the device: one array goes up, three come down). The arrays are cut
+ * into pieces of 16 MiB per array; each piece is copied into a ring of four device stages (three piece buffers
  * each: 192 MiB of device memory whatever n is, so the arrays may be far larger than the device's
  * memory), run through the five kernels and copied back on three streams of the library's own, so
  * that uploads, kernels and downloads of different pieces overlap and both directions of the host

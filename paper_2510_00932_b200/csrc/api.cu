@@ -375,7 +375,8 @@ int run_op(int op, int dtype, const void *x, const void *y, void *out, double sc
 }
 
 // Host-buffer pass, pipelined through a small ring of device buffers: the arrays are cut into pieces
-// of g_chain_piece_bytes per array; piece k is uploaded into ring stage k mod kChainRing on one
+// of g_chain_piece_bytes per array; piece k of a (the pass's only input: b and c are overwritten before
+// they are read) is uploaded into ring stage k mod kChainRing on one
 // stream, run through the five kernels on a second (Dot as a double partial sum per piece), and
 // downloaded on a third, so that uploads, kernels and downloads of different pieces overlap and the
 // two directions of the host link are busy at the same time. A stage is refilled only after the
@@ -437,8 +438,9 @@ int chain_host(T *a, T *b, T *c, double scalar, size_t n, T *dot_out) {
             // the stage is free once the download of its previous piece (this call's or an earlier
             // call's) has finished; an event that was never recorded counts as complete
             if ((e = cudaStreamWaitEvent(up, d->chain_downloaded[s], 0)) != cudaSuccess) return cuda_fail(e);
-            for (int i = 0; i < 3; ++i)
-                if ((e = cudaMemcpyAsync(dev[i], host[i] + lo, len * sizeof(T), cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e);
+            // only a travels to the device: the pass overwrites c (c <- a) and b (b <- s*c) before it reads
+            // them, so their contents on entry are no inputs of the computation
+            if ((e = cudaMemcpyAsync(dev[0], host[0] + lo, len * sizeof(T), cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaEventRecord(d->chain_uploaded[s], up)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaStreamWaitEvent(run, d->chain_uploaded[s], 0)) != cudaSuccess) return cuda_fail(e);
             T *pa = dev[0], *pb = dev[1], *pc = dev[2];

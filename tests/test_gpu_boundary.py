@@ -183,6 +183,12 @@ def test_host_arrays_many_times_larger_than_the_device_ring(so, torch, oracle, t
     oa, ob, oc, od = oracle.chain(a, b, c, scalar)
     assert_bits_equal(ha, oa, "a"); assert_bits_equal(hb, ob, "b"); assert_bits_equal(hc, oc, "c")
     assert abs(float(d) - od) <= (1e-12 if t == "f64" else 1e-5) * abs(od)
+    # b and c are outputs only (the dataflow overwrites them before reading them): whatever they hold on
+    # entry, NaN included, the results are the same
+    ha, hb, hc = a.copy(), np.full_like(b, np.nan), np.full_like(c, np.nan)
+    d2 = so.chain_host(ha, hb, hc, scalar)
+    assert_bits_equal(ha, oa, "a"); assert_bits_equal(hb, ob, "b"); assert_bits_equal(hc, oc, "c")
+    assert np.array([d2]).tobytes() == np.array([d]).tobytes()
 
 
 def test_host_entry_point_from_two_threads(so, torch, oracle):
