@@ -258,7 +258,8 @@ bool valid_tuning(const streamops_tuning_t &t) {
 // Picks the workspace slot of one Dot call on `stream` and fills in its scratch pointers.
 // Ordinary calls: the slot this stream used last (stream order makes reuse safe), else a slot never
 // used, else a slot whose last Dot has finished (the ticket words are copied to the host on a stream
-// of the library's own: this is the only path that waits for anything, and only for that copy); if all kDotLiveSlots slots are still in flight on other streams, STREAMOPS_ERR_WORKSPACE.
+// of the library's own: this is the only path that waits for anything, and only for that copy); if
+// all kDotLiveSlots slots are still in flight on other streams, STREAMOPS_ERR_WORKSPACE.
 // Calls made while `stream` is being captured: one of the kDotCaptureSlots slots set aside for graphs,
 // handed out in turn and never shared with ordinary calls; the slot is baked into the graph.
 int acquire_dot_slot(DeviceState *d, cudaStream_t stream, DotScratch *scratch, DotSlot **live) {
