@@ -110,6 +110,18 @@ int stream_dot_wide_f32(const float *x, const float *y, double *out, double scal
 int stream_fold_f64(const double *partials, double *out, double scalar, size_t count, streamops_stream_t stream);
 int stream_fold_f32(const double *partials, float *out, double scalar, size_t count, streamops_stream_t stream);
 
+/* The default double-precision Dot (same kernel, launch shape and result as stream_dot_f64 under the default
+ * tuning) instrumented for profiling: thread 0 of block b stores three readings of the GPU's global
+ * nanosecond timer into stamps[3 b .. 3 b + 2] -- after the wait for the previous kernel of the stream, after
+ * the block's last multiply-add (all its data has arrived), and at the block's end (for the block that
+ * finishes the Dot: after the final fold and the write of out[0]). stamps is a DEVICE array of at least
+ * 3 * STREAMOPS_TIMELINE_MAX_BLOCKS entries; *blocks (HOST) receives the number of blocks launched. x and y
+ * must be 32-byte aligned and n > 0 (STREAMOPS_ERR_ARG otherwise). `python -m paper_2510_00932_b200.timeline`
+ * turns the stamps into a timeline of one launch inside a train of launches. */
+int stream_dot_timeline_f64(const double *x, const double *y, double *out, size_t n, streamops_stream_t stream,
+                            unsigned long long *stamps, unsigned *blocks);
+#define STREAMOPS_TIMELINE_MAX_BLOCKS 1024
+
 /* Dot without any allocation (the paper has no counterpart; this entry point exists for callers
  * that cannot allocate device memory when they need the result: code that runs after a memory
  * pool has taken the whole device, loops that must not take the allocator's lock or trigger its

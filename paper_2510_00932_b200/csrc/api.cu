@@ -522,6 +522,34 @@ STREAMOPS_BINARY(stream_triad_f32, OP_TRIAD, float, DT_F32)
 STREAMOPS_BINARY(stream_dot_f64, OP_DOT, double, DT_F64)
 STREAMOPS_BINARY(stream_dot_f32, OP_DOT, float, DT_F32)
 
+int stream_dot_timeline_f64(const double *x, const double *y, double *out, size_t n, streamops_stream_t stream_,
+                            unsigned long long *stamps, unsigned *blocks) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!stamps || !blocks) return STREAMOPS_ERR_NULL;
+    int status = check_args(OP_DOT, 8, x, y, out, n, 8);
+    if (status != STREAMOPS_OK) return status;
+    if (n == 0 || (((uintptr_t)x | (uintptr_t)y) & 31)) return STREAMOPS_ERR_ARG;     // the 32-byte-vector kernel only
+    DeviceState *d = nullptr;
+    if ((status = current_device_state(&d)) != STREAMOPS_OK) return status;
+    streamops_tuning_t t = default_tuning(OP_DOT, DT_F64);
+    const VecLaunch c = resolve_vec(t, *d, OP_DOT, 8, x, y, out, n);
+    if (c.grid > (unsigned)STREAMOPS_TIMELINE_MAX_BLOCKS) return STREAMOPS_ERR_ARG;
+    DotScratch scratch{nullptr, nullptr, 0};
+    DotSlot *live_slot = nullptr;
+    if ((status = acquire_dot_slot(d, stream, &scratch, &live_slot)) != STREAMOPS_OK) return status;
+    const cudaError_t e = launch_dot_timeline(c, x, y, out, n, scratch, stamps, stream);
+    if (e != cudaSuccess) {
+        if (live_slot) {
+            std::lock_guard<std::mutex> lock(d->slot_mutex);
+            --live_slot->issued;
+        }
+        return cuda_fail(e);
+    }
+    *blocks = c.grid;
+    g_launches.fetch_add(1);
+    return STREAMOPS_OK;
+}
+
 int stream_dot_wide_f32(const float *x, const float *y, double *out, double scalar, size_t n, streamops_stream_t stream) {
     return run_op(OP_DOT, DT_F32, x, y, out, scalar, n, stream, true);
 }

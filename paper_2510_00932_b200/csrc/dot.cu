@@ -94,14 +94,27 @@ dot_pass1_kernel(const T *x, const T *y, size_t n, double *partials, unsigned lo
     publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, seq);
 }
 
+__device__ __forceinline__ unsigned long long global_nanoseconds() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
 // Rolling-slot pass 1 (see the file comment). A tile is blockDim.x vectors: one vector per thread.
-template <typename T, int VB, int S, int POL, bool SINGLE_LAUNCH>
+// With TRACE (the timeline entry point only) thread 0 of every block stores three global-timer readings
+// into stamps[3 * blockIdx.x ..]: after the wait for the previous kernel, after its last fold, and at the
+// block's end (for the finishing block: after the final fold and the write of the result).
+template <typename T, int VB, int S, int POL, bool SINGLE_LAUNCH, bool TRACE = false>
 __global__ void __launch_bounds__(kMaxThreads, S <= 2 ? 2 : 1)
-dot_roll_kernel(const T *x, const T *y, size_t n, double *partials, unsigned long long *ticket, T *out, unsigned seq) {
+dot_roll_kernel(const T *x, const T *y, size_t n, double *partials, unsigned long long *ticket, T *out, unsigned seq,
+                unsigned long long *stamps) {
     constexpr int EPV = VB / (int)sizeof(T);
     __shared__ double warp_part[32];
     __shared__ bool is_last;
     grid_dependency_sync();
+    if constexpr (TRACE) {
+        if (threadIdx.x == 0) stamps[3 * blockIdx.x] = global_nanoseconds();
+    }
     const char *xb = reinterpret_cast<const char *>(x);
     const char *yb = reinterpret_cast<const char *>(y);
     const uint64_t l2pol = make_l2_policies<POL>().ld;
@@ -155,8 +168,14 @@ dot_roll_kernel(const T *x, const T *y, size_t n, double *partials, unsigned lon
     double tsum = acc[0];
 #pragma unroll
     for (int s = 1; s < S; ++s) tsum += acc[s];
+    if constexpr (TRACE) {
+        if (threadIdx.x == 0) stamps[3 * blockIdx.x + 1] = global_nanoseconds();
+    }
     const double bsum = block_sum(tsum, warp_part);
     publish_partial<T, SINGLE_LAUNCH>(bsum, partials, ticket, out, warp_part, &is_last, seq);
+    if constexpr (TRACE) {
+        if (threadIdx.x == 0) stamps[3 * blockIdx.x + 2] = global_nanoseconds();
+    }
 }
 
 template <typename T>
@@ -197,7 +216,7 @@ cudaError_t launch_pol(const VecLaunch &c, const T *x, const T *y, size_t n, con
 template <typename T, int VB, bool SL>
 cudaError_t launch_roll(const VecLaunch &c, const T *x, const T *y, size_t n, const DotScratch &s, T *out, cudaStream_t st) {
     const bool plain = c.policy == 0;
-#define STREAMOPS_ROLL(S, P) launch_kernel(dot_roll_kernel<T, VB, S, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, s.seq)
+#define STREAMOPS_ROLL(S, P) launch_kernel(dot_roll_kernel<T, VB, S, P, SL>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n, s.partials, s.ticket, out, s.seq, (unsigned long long *)nullptr)
     if (c.unroll == 2) return plain ? STREAMOPS_ROLL(2, 0) : STREAMOPS_ROLL(2, 4);
     if (c.unroll == 4) return plain ? STREAMOPS_ROLL(4, 0) : STREAMOPS_ROLL(4, 4);
 #undef STREAMOPS_ROLL
@@ -263,6 +282,13 @@ cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, bool wide
                                     scratch, stream, launches);
     return launch_dot_t<float>(cfg, two_pass, wide, (const float *)x, (const float *)y, out, n,
                                scratch, stream, launches);
+}
+
+// The default double-precision Dot (two rolling slots, evict-first loads, single launch) with time stamps.
+cudaError_t launch_dot_timeline(const VecLaunch &c, const double *x, const double *y, double *out, size_t n,
+                                const DotScratch &s, unsigned long long *stamps, cudaStream_t st) {
+    return launch_kernel(dot_roll_kernel<double, 32, 2, 4, true, true>, c.grid, c.threads, 0, st, c.pdl != 0, x, y, n,
+                         s.partials, s.ticket, out, s.seq, stamps);
 }
 
 cudaError_t launch_fold(int dtype, const double *partials, size_t count, void *out, cudaStream_t stream) {

@@ -92,6 +92,9 @@ cudaError_t launch_elementwise(int op, int dtype, const VecLaunch &cfg, const vo
 cudaError_t launch_dot(int dtype, const VecLaunch &cfg, bool two_pass, bool wide, const void *x, const void *y,
                        void *out, size_t n, const DotScratch &scratch, cudaStream_t stream,
                        int *launches);
+// the default double-precision Dot with three time stamps per block (see stream_dot_timeline_f64)
+cudaError_t launch_dot_timeline(const VecLaunch &cfg, const double *x, const double *y, double *out, size_t n,
+                                const DotScratch &scratch, unsigned long long *stamps, cudaStream_t stream);
 // dot_comp.cu: Dot with (sum, error) pairs throughout; one launch; cfg.grid <= kMaxDotBlocks / 2
 cudaError_t launch_dot_compensated(int dtype, const VecLaunch &cfg, const void *x, const void *y, void *out, size_t n,
                                    const DotScratch &scratch, cudaStream_t stream);

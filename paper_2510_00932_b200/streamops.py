@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         for t in ("f32", "f64"):
             f = getattr(L, f"stream_fold_{t}")
             f.argtypes, f.restype = [vp, vp, dbl, sz, vp], ci
+        L.stream_dot_timeline_f64.argtypes = [vp, vp, vp, sz, vp, vp, ctypes.POINTER(ctypes.c_uint)]
+        L.stream_dot_timeline_f64.restype = ci
         L.stream_dot_noalloc_f64.argtypes, L.stream_dot_noalloc_f64.restype = [vp, vp, vp, dbl, sz, vp], ci
         L.shmem_mix_u32.argtypes, L.shmem_mix_u32.restype = [vp, vp, ctypes.c_uint, sz, vp], ci
         L.streamops_set_shmem_width.argtypes, L.streamops_set_shmem_width.restype = [ci], ci
@@ -212,6 +214,24 @@ def fold(partials, out):
         raise ValueError("fold writes one element on the device that holds the partial sums")
     _raise(getattr(lib(), f"stream_fold_{suf}")(partials.data_ptr(), out.data_ptr(), 0.0, partials.numel(), stream))
     return out
+
+
+TIMELINE_MAX_BLOCKS = 1024
+
+
+def dot_timeline(x, y, out, stamps) -> int:
+    """The default fp64 Dot with three global-timer stamps per block written to the int64 device tensor
+    `stamps` (at least 3 * TIMELINE_MAX_BLOCKS entries); returns the number of blocks launched."""
+    import torch
+    suf, stream = _marshal(x, y, out)
+    if suf != "f64" or x.numel() != y.numel() or out.numel() != 1:
+        raise ValueError("dot_timeline takes two equal-length float64 inputs and a one-element output")
+    if stamps.dtype != torch.int64 or not stamps.is_cuda or stamps.numel() < 3 * TIMELINE_MAX_BLOCKS or not stamps.is_contiguous():
+        raise ValueError("stamps is a contiguous int64 CUDA tensor of at least 3 * TIMELINE_MAX_BLOCKS entries")
+    blocks = ctypes.c_uint(0)
+    _raise(lib().stream_dot_timeline_f64(x.data_ptr(), y.data_ptr(), out.data_ptr(), x.numel(), stream, stamps.data_ptr(),
+                                         ctypes.byref(blocks)))
+    return int(blocks.value)
 
 
 DOT_NOALLOC_MAX_N = 1 << 28

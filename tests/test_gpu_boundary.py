@@ -222,3 +222,28 @@ def test_binding_refuses_tensors_of_a_device_that_is_not_current(so, torch):
     torch.cuda.set_device(0)
     with pytest.raises(ValueError):
         so.copy(x, x.clone())
+
+
+def test_instrumented_dot_returns_the_ordinary_bits_and_ordered_time_stamps(so, torch):
+    """stream_dot_timeline_f64 is the default fp64 Dot plus three timer readings per block: same bits
+    as stream_dot_f64, stamps non-decreasing within a block, the finishing block the last to end."""
+    n = (1 << 23) + 12
+    rng = np.random.Generator(np.random.PCG64(131))
+    x, y = (torch.from_numpy(rng.standard_normal(n)).cuda() for _ in range(2))
+    out, ref = (torch.zeros(1, dtype=torch.float64, device="cuda") for _ in range(2))
+    stamps = torch.zeros(3 * so.TIMELINE_MAX_BLOCKS, dtype=torch.int64, device="cuda")
+    so.dot(x, y, ref)
+    blocks = so.dot_timeline(x, y, out, stamps)
+    torch.cuda.synchronize()
+    assert out.cpu().numpy().tobytes() == ref.cpu().numpy().tobytes()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert blocks == 2 * sms
+    t = stamps[:3 * blocks].cpu().numpy().reshape(blocks, 3)
+    assert (t[:, 0] > 0).all() and (t[:, 0] <= t[:, 1]).all() and (t[:, 1] <= t[:, 2]).all()
+    assert t[:, 2].max() - t[:, 0].min() < 5_000_000                      # a few hundred microseconds at most, in ns
+    assert (stamps[3 * blocks:] == 0).all()
+    L = so.lib()
+    import ctypes
+    b = ctypes.c_uint(0)
+    assert L.stream_dot_timeline_f64(x[1:].data_ptr(), y[1:].data_ptr(), out.data_ptr(), n - 1, None, stamps.data_ptr(), ctypes.byref(b)) == 7
+    assert L.stream_dot_timeline_f64(x.data_ptr(), y.data_ptr(), out.data_ptr(), n, None, None, ctypes.byref(b)) == 1
